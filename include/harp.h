@@ -1,0 +1,125 @@
+/* harp.h -- C ABI of the B200 (sm_100a) HARP apply library.
+ *
+ * A HARP processor is the orthogonal map (row-vector convention, y = x Q)
+ *
+ *     Q = D_s . Pi . T,      T = M_0 . M_1 ... M_{m-1}
+ *
+ * D_s : Rademacher sign diagonal (paper, Section "HARP processors": sign flips as in
+ *       RHT preprocessing; Assumption 1(d): applied as diagonal matrices).
+ * Pi  : a fixed permutation, applied as a gather v_i = u_{perm[i]} (the "fixed
+ *       permutation convention" of Theorem 1).
+ * M_t : stride stage t of Eq. 7 with the Mixed-Radix schedule of Eq. 6:
+ *       s_t = prod_{j<t} b_j, g = d/(b_t s_t); for every (alpha < g, beta < s_t) the b_t
+ *       coordinates {alpha b_t s_t + r s_t + beta : r < b_t} (Lemma 1) are multiplied on
+ *       the right by block kernel K_t[c], c = alpha s_t + beta:
+ *           out[base + j s_t] = sum_i in[base + i s_t] * K_t[c][i][j].
+ *       Stage 0 (stride 1) is applied first (Algorithm 1, Eq. 8).
+ *
+ * All functions return a status, never throw and never abort; nothing is launched on
+ * invalid input.  Pointers are marked HOST or DEVICE.  Device buffers are caller-owned and
+ * contiguous row-major; results overwrite the input.  A buffer must be aligned to its
+ * element size (else HARP_ERR_BAD_DIM); the fast kernels additionally need a 16-byte
+ * aligned base, and a call that lacks it runs on the generic kernel.
+ * The library never falls back to a CPU path: unsupported shapes return
+ * HARP_ERR_UNSUPPORTED.
+ */
+#ifndef HARP_H_
+#define HARP_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct harp_plan harp_plan_t; /* opaque; immutable after create */
+
+typedef enum {
+    HARP_OK = 0,
+    HARP_ERR_NULL = 1,          /* a required pointer is NULL                         */
+    HARP_ERR_BAD_DIM = 2,       /* d < 2, n_rows < 0, or d too large                  */
+    HARP_ERR_BAD_SCHEDULE = 3,  /* n_stages < 1, a radix < 2, or prod(radices) != d   */
+    HARP_ERR_BAD_PERM = 4,      /* perm is not a bijection of 0..d-1                  */
+    HARP_ERR_BAD_SIGNS = 5,     /* a sign is not +1 or -1                             */
+    HARP_ERR_BAD_DTYPE = 6,
+    HARP_ERR_DIM_MISMATCH = 7,
+    HARP_ERR_UNSUPPORTED = 8,   /* valid input this build has no kernel for           */
+    HARP_ERR_ALLOC = 9,         /* host or device allocation failed                   */
+    HARP_ERR_CUDA = 10,         /* a CUDA runtime call or launch failed               */
+    HARP_ERR_TOO_LARGE = 11     /* exceeds a documented fixed capacity                */
+} harp_status_t;
+
+typedef enum { HARP_F32 = 0, HARP_BF16 = 1 } harp_dtype_t;
+
+/* Kernel families; HARP_KERNEL_AUTO lets the library choose. */
+typedef enum { HARP_KERNEL_AUTO = 0, HARP_KERNEL_GENERIC = 1, HARP_KERNEL_FAST = 2 } harp_kernel_t;
+
+/* Build a processor (Eq. 6-9 of the paper; Algorithm 1 lines 2 and 7-8 for the stride
+ * and block-kernel layout).
+ *   out      HOST  receives the plan; untouched on error
+ *   d        transformed dimension, 2 <= d <= 2^20
+ *   n_stages m >= 1;  radices HOST int32[m], each >= 2, product == d
+ *   perm     HOST int32[d] bijection, forward gathers v[i] = u[perm[i]]; NULL = identity
+ *   signs    HOST int8[d] with entries +1/-1;  NULL = all +1
+ *   blocks   HOST array of m pointers; blocks[t] = float[d/b_t][b_t][b_t] row-major
+ * Every host array is copied; the plan owns its device copies on the current CUDA
+ * device.  Orthogonality of the blocks is not checked: the library applies what it is
+ * given.  Validation happens before the first CUDA call. */
+harp_status_t harp_plan_create(harp_plan_t **out, int64_t d, int32_t n_stages,
+                               const int32_t *radices, const int32_t *perm,
+                               const int8_t *signs, const float *const *blocks);
+
+/* Release the plan and its device memory.  NULL is allowed. */
+void harp_plan_destroy(harp_plan_t *plan);
+
+/* d of the plan, or -1 for NULL. */
+int64_t harp_plan_dim(const harp_plan_t *plan);
+
+/* Apply the processor to a batch of rows, in place (Algorithm 1: y = x T(Theta), with
+ * the sign diagonal and permutation in front; transpose != 0 applies Q^T, the map used
+ * on the output side of a layer, W^ = U W~^ V^T).
+ *   x        DEVICE n_rows x d, dtype fp32 or bf16, overwritten with the result
+ *   stream   a cudaStream_t passed as void* (NULL = default stream)
+ * Asynchronous on stream; does not synchronise.  n_rows == 0 returns HARP_OK without
+ * a launch.  bf16 results are rounded once, to nearest even, at the store. */
+harp_status_t harp_apply(const harp_plan_t *plan, void *x, int64_t n_rows, harp_dtype_t dtype,
+                         int transpose, void *stream);
+
+/* Same as harp_apply with an explicit kernel family (tests and benchmarks).
+ * Returns HARP_ERR_UNSUPPORTED if that family has no kernel for this plan/dtype. */
+harp_status_t harp_apply_ex(const harp_plan_t *plan, void *x, int64_t n_rows,
+                            harp_dtype_t dtype, int transpose, harp_kernel_t kernel,
+                            void *stream);
+
+/* Two-sided processing of a weight matrix, W <- Q_out^T W Q_in (paper, Section
+ * "Incoherence processing": W~ = U^T W V with U = Q_out, V = Q_in; Algorithm 3 line 3).
+ *   W        DEVICE d_out x d_in row-major, d_out = dim(plan_out), d_in = dim(plan_in)
+ *   scratch  DEVICE buffer of harp_two_sided_scratch_bytes(...) bytes, 256-byte aligned,
+ *            or NULL to let the call allocate and free it on the stream
+ *            (cudaMallocAsync/cudaFreeAsync).
+ * Asynchronous on stream. */
+harp_status_t harp_apply_two_sided(void *W, harp_dtype_t dtype, const harp_plan_t *plan_out,
+                                   const harp_plan_t *plan_in, void *scratch, void *stream);
+
+/* Bytes of scratch harp_apply_two_sided needs for these plans and dtype (0 on bad input). */
+int64_t harp_two_sided_scratch_bytes(const harp_plan_t *plan_out, const harp_plan_t *plan_in,
+                                     harp_dtype_t dtype);
+
+/* Apply to rows that live in HOST memory (pinned memory gives full copy speed):
+ * copies chunks host->device, applies, copies back, on two internal streams so that
+ * copies overlap kernels; returns after the last copy has completed.  The device staging
+ * buffers belong to the plan and are created at the first call.
+ *   x_host   HOST n_rows x d, overwritten with the result */
+harp_status_t harp_apply_host(harp_plan_t *plan, void *x_host, int64_t n_rows,
+                              harp_dtype_t dtype, int transpose);
+
+/* Number of kernels this library has launched in the calling process (all plans). */
+int64_t harp_launch_count(void);
+
+/* Static, human-readable text for a status. */
+const char *harp_status_string(harp_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HARP_H_ */

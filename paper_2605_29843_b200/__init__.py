@@ -1,0 +1,175 @@
+"""B200-native HARP apply: thin ctypes binding over libharp.so.
+
+The functions here carry the same names as the C ABI in ``include/harp.h`` and do
+argument marshalling only; every step of the path runs in the CUDA library.  There is
+no CPU fallback: if the library is missing or fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libharp.so")
+
+HARP_F32, HARP_BF16 = 0, 1
+KERNEL_AUTO, KERNEL_GENERIC, KERNEL_FAST = 0, 1, 2
+HARP_OK = 0
+HARP_ERR_UNSUPPORTED = 8
+
+_lib: Optional[ctypes.CDLL] = None
+
+
+class HarpError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = int(status)
+        super().__init__(f"{what}: {status_string(status)} (status {status})")
+
+
+def lib() -> ctypes.CDLL:
+    """Load libharp.so (built in-tree by ``paper_2605_29843_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not found: run `python -m paper_2605_29843_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i64, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32
+        L.harp_plan_create.restype = ctypes.c_int
+        L.harp_plan_create.argtypes = [ctypes.POINTER(vp), i64, i32, vp, vp, vp, ctypes.POINTER(vp)]
+        L.harp_plan_destroy.restype = None
+        L.harp_plan_destroy.argtypes = [vp]
+        L.harp_plan_dim.restype = i64
+        L.harp_plan_dim.argtypes = [vp]
+        L.harp_apply.restype = ctypes.c_int
+        L.harp_apply.argtypes = [vp, vp, i64, ctypes.c_int, ctypes.c_int, vp]
+        L.harp_apply_ex.restype = ctypes.c_int
+        L.harp_apply_ex.argtypes = [vp, vp, i64, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp]
+        L.harp_apply_two_sided.restype = ctypes.c_int
+        L.harp_apply_two_sided.argtypes = [vp, ctypes.c_int, vp, vp, vp, vp]
+        L.harp_two_sided_scratch_bytes.restype = i64
+        L.harp_two_sided_scratch_bytes.argtypes = [vp, vp, ctypes.c_int]
+        L.harp_apply_host.restype = ctypes.c_int
+        L.harp_apply_host.argtypes = [vp, vp, i64, ctypes.c_int, ctypes.c_int]
+        L.harp_launch_count.restype = i64
+        L.harp_launch_count.argtypes = []
+        L.harp_status_string.restype = ctypes.c_char_p
+        L.harp_status_string.argtypes = [ctypes.c_int]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().harp_status_string(int(status)).decode()
+
+
+def harp_launch_count() -> int:
+    return int(lib().harp_launch_count())
+
+
+class Plan:
+    """Owner of a ``harp_plan_t*``; destroyed with the object."""
+
+    def __init__(self, handle: int, d: int):
+        self.handle = handle
+        self.d = d
+
+    def __del__(self):
+        h, self.handle = getattr(self, "handle", None), None
+        if h and _lib is not None:
+            _lib.harp_plan_destroy(h)
+
+
+def harp_plan_create_status(d: int, radices: Sequence[int], perm, signs, blocks):
+    """Raw call: returns (status, Plan or None).  Arrays are host numpy arrays."""
+    L = lib()
+    rad = np.ascontiguousarray(radices, dtype=np.int32)
+    pm = None if perm is None else np.ascontiguousarray(perm, dtype=np.int32)
+    sg = None if signs is None else np.ascontiguousarray(signs, dtype=np.int8)
+    blks = [np.ascontiguousarray(b, dtype=np.float32) for b in blocks] if blocks is not None else None
+    if blks is not None:
+        arr = (ctypes.c_void_p * max(1, len(blks)))(*[b.ctypes.data for b in blks])
+    else:
+        arr = None
+    out = ctypes.c_void_p()
+    st = L.harp_plan_create(ctypes.byref(out), int(d), len(rad), rad.ctypes.data,
+                            None if pm is None else pm.ctypes.data,
+                            None if sg is None else sg.ctypes.data, arr)
+    if st != HARP_OK:
+        return st, None
+    return st, Plan(out.value, int(d))
+
+
+def harp_plan_create(d: int, radices: Sequence[int], perm=None, signs=None, blocks=None) -> Plan:
+    st, plan = harp_plan_create_status(d, radices, perm, signs, blocks)
+    if st != HARP_OK:
+        raise HarpError(st, "harp_plan_create")
+    return plan
+
+
+def plan_from_spec(spec) -> Plan:
+    """Plan from a ``workloads.PlanSpec``-like object (d, radices, perm, signs, blocks)."""
+    return harp_plan_create(spec.d, spec.radices, spec.perm, spec.signs, spec.blocks)
+
+
+def harp_plan_dim(plan: Plan) -> int:
+    return int(lib().harp_plan_dim(plan.handle))
+
+
+def harp_apply(plan: Plan, x_ptr: int, n_rows: int, dtype: int, transpose: bool = False,
+               stream: int = 0, kernel: int = KERNEL_AUTO) -> None:
+    """x_ptr: device address of n_rows x d elements, transformed in place on ``stream``."""
+    st = lib().harp_apply_ex(plan.handle, x_ptr, int(n_rows), int(dtype), 1 if transpose else 0,
+                             int(kernel), stream or None)
+    if st != HARP_OK:
+        raise HarpError(st, "harp_apply")
+
+
+def harp_apply_two_sided(w_ptr: int, dtype: int, plan_out: Plan, plan_in: Plan,
+                         scratch_ptr: int = 0, stream: int = 0) -> None:
+    st = lib().harp_apply_two_sided(w_ptr, int(dtype), plan_out.handle, plan_in.handle,
+                                    scratch_ptr or None, stream or None)
+    if st != HARP_OK:
+        raise HarpError(st, "harp_apply_two_sided")
+
+
+def harp_two_sided_scratch_bytes(plan_out: Plan, plan_in: Plan, dtype: int) -> int:
+    return int(lib().harp_two_sided_scratch_bytes(plan_out.handle, plan_in.handle, int(dtype)))
+
+
+def harp_apply_host(plan: Plan, host_ptr: int, n_rows: int, dtype: int, transpose: bool = False) -> None:
+    """host_ptr: host address (pinned for full speed) of n_rows x d elements, in place."""
+    st = lib().harp_apply_host(plan.handle, host_ptr, int(n_rows), int(dtype), 1 if transpose else 0)
+    if st != HARP_OK:
+        raise HarpError(st, "harp_apply_host")
+
+
+# ---- torch conveniences (device memory and streams only) ----
+
+def _torch_dtype_code(t) -> int:
+    import torch
+    if t.dtype == torch.float32:
+        return HARP_F32
+    if t.dtype == torch.bfloat16:
+        return HARP_BF16
+    raise TypeError(f"unsupported dtype {t.dtype}")
+
+
+def apply_(plan: Plan, x, transpose: bool = False, kernel: int = KERNEL_AUTO):
+    """In-place apply to a contiguous CUDA tensor [n_rows, d] on torch's current stream."""
+    import torch
+    assert x.is_cuda and x.is_contiguous() and x.dim() == 2 and x.shape[1] == plan.d
+    harp_apply(plan, x.data_ptr(), x.shape[0], _torch_dtype_code(x), transpose,
+               torch.cuda.current_stream().cuda_stream, kernel)
+    return x
+
+
+def two_sided_(w, plan_out: Plan, plan_in: Plan, scratch=None):
+    import torch
+    assert w.is_cuda and w.is_contiguous() and w.shape == (plan_out.d, plan_in.d)
+    harp_apply_two_sided(w.data_ptr(), _torch_dtype_code(w), plan_out, plan_in,
+                         0 if scratch is None else scratch.data_ptr(),
+                         torch.cuda.current_stream().cuda_stream)
+    return w

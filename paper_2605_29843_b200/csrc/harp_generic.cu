@@ -1,0 +1,149 @@
+// Generic CUDA-core kernel: any schedule, any radix, fp32 arithmetic.
+//
+// One CTA owns a tile of R whole rows in shared memory (fp32) for all stages, so a
+// row is read from HBM once and written once.  A work item is one output
+// coordinate of one row; every thread computes its items of a stage into
+// registers, the CTA synchronises, the items are written back in place, and the
+// next stage starts.  Block kernels are read through the read-only path from L2.
+// This path defines correct behaviour for every plan the ABI accepts (up to the
+// shared-memory capacity); the tensor-core path in harp_fast.cu is faster where
+// it applies.
+#include "harp_internal.h"
+
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kMaxItems = 32;   // R*d <= kThreads*kMaxItems
+
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+template <typename T, int ITEMS>
+__global__ void __launch_bounds__(kThreads, 1)
+harp_generic_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_cta, StageTable st,
+                    const float *__restrict__ blocks, const int32_t *__restrict__ perm,
+                    const int8_t *__restrict__ signs, int transpose) {
+    extern __shared__ float v[];                     // [rows_per_cta][d]
+    const int64_t row0 = (int64_t)blockIdx.x * rows_per_cta;
+    const int rows = (int)min((int64_t)rows_per_cta, n_rows - row0);
+    const int total = rows * d;
+    T *xt = x + row0 * d;
+
+    // a1-a3: load, sign, gather (forward) -- or plain load (transpose)
+    for (int idx = threadIdx.x; idx < total; idx += kThreads) {
+        const int r = idx / d, i = idx - r * d;
+        if (!transpose) {
+            const int src = perm ? perm[i] : i;
+            float val = to_f32<T>(xt[(int64_t)r * d + src]);
+            if (signs && signs[src] < 0) val = -val;
+            v[idx] = val;
+        } else {
+            v[idx] = to_f32<T>(xt[idx]);
+        }
+    }
+    __syncthreads();
+
+    // a4 / a6: stages 0..m-1 (forward) or m-1..0 with transposed kernels
+    for (int k = 0; k < st.m; ++k) {
+        const int t = transpose ? st.m - 1 - k : k;
+        const int b = st.b[t], s = st.s[t];
+        const int bs = b * s;
+        const float *Kt = blocks + st.off[t];
+        float acc[ITEMS];
+#pragma unroll
+        for (int it = 0; it < ITEMS; ++it) {
+            const int idx = threadIdx.x + it * kThreads;
+            acc[it] = 0.f;
+            if (idx < total) {
+                const int r = idx / d, p = idx - r * d;
+                const int alpha = p / bs, rem = p - alpha * bs;
+                const int j = rem / s, beta = rem - j * s;
+                const int c = alpha * s + beta;
+                const float *Kc = Kt + (int64_t)c * b * b;
+                const float *vin = v + r * d + alpha * bs + beta;
+                float a = 0.f;
+                if (!transpose) {
+                    for (int i = 0; i < b; ++i) a = fmaf(vin[i * s], __ldg(Kc + i * b + j), a);
+                } else {
+                    for (int i = 0; i < b; ++i) a = fmaf(vin[i * s], __ldg(Kc + j * b + i), a);
+                }
+                acc[it] = a;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int it = 0; it < ITEMS; ++it) {
+            const int idx = threadIdx.x + it * kThreads;
+            if (idx < total) v[idx] = acc[it];
+        }
+        __syncthreads();
+    }
+
+    // a5: store -- or scatter and sign (transpose)
+    for (int idx = threadIdx.x; idx < total; idx += kThreads) {
+        const int r = idx / d, i = idx - r * d;
+        if (!transpose) {
+            xt[idx] = from_f32<T>(v[idx]);
+        } else {
+            const int dst = perm ? perm[i] : i;
+            float val = v[idx];
+            if (signs && signs[dst] < 0) val = -val;
+            xt[(int64_t)r * d + dst] = from_f32<T>(val);
+        }
+    }
+}
+
+template <typename T, int ITEMS>
+harp_status_t launch(const harp_plan *plan, void *x, int64_t n_rows, int rows_per_cta, int transpose,
+                     cudaStream_t stream) {
+    auto kern = harp_generic_kernel<T, ITEMS>;
+    const size_t smem = (size_t)rows_per_cta * plan->d * sizeof(float);
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+        return HARP_ERR_CUDA;
+    const int64_t grid = (n_rows + rows_per_cta - 1) / rows_per_cta;
+    if (grid > 0x7fffffffLL) return HARP_ERR_BAD_DIM;
+    kern<<<(unsigned)grid, kThreads, smem, stream>>>((T *)x, n_rows, (int)plan->d, rows_per_cta, plan->st,
+                                                      plan->d_blocks, plan->d_perm, plan->d_signs, transpose);
+    g_harp_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? HARP_OK : HARP_ERR_CUDA;
+}
+
+}  // namespace
+
+harp_status_t harp_generic_supported(const harp_plan *plan, harp_dtype_t dtype) {
+    (void)dtype;
+    if (plan->d > (int64_t)kThreads * kMaxItems) return HARP_ERR_UNSUPPORTED;
+    if ((size_t)plan->d * sizeof(float) > 227u * 1024u) return HARP_ERR_UNSUPPORTED;
+    return HARP_OK;
+}
+
+harp_status_t harp_generic_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype,
+                                 int transpose, cudaStream_t stream) {
+    harp_status_t ok = harp_generic_supported(plan, dtype);
+    if (ok != HARP_OK) return ok;
+    const int64_t d = plan->d;
+    // rows per CTA: as many as registers (kMaxItems) and shared memory allow, at most 8,
+    // but keep at least ~2 CTAs per SM in flight when the batch is small.
+    int r = (int)((int64_t)kThreads * kMaxItems / d);
+    const int r_smem = (int)((227 * 1024) / (d * (int64_t)sizeof(float)));
+    if (r > r_smem) r = r_smem;
+    if (r > 8) r = 8;
+    while (r > 1 && (n_rows + r - 1) / r < 296) --r;
+    if (r < 1) r = 1;
+    const int64_t items = ((int64_t)r * d + kThreads - 1) / kThreads;
+#define HARP_GEN_DISPATCH(T)                                                                  \
+    if (items <= 4) return launch<T, 4>(plan, x, n_rows, r, transpose, stream);               \
+    if (items <= 8) return launch<T, 8>(plan, x, n_rows, r, transpose, stream);               \
+    if (items <= 16) return launch<T, 16>(plan, x, n_rows, r, transpose, stream);             \
+    return launch<T, 32>(plan, x, n_rows, r, transpose, stream);
+    if (dtype == HARP_F32) {
+        HARP_GEN_DISPATCH(float)
+    } else {
+        HARP_GEN_DISPATCH(__nv_bfloat16)
+    }
+#undef HARP_GEN_DISPATCH
+}

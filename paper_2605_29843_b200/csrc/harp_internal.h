@@ -1,0 +1,61 @@
+// Internal declarations shared by the translation units of libharp.so.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+#include <vector>
+
+#include "harp.h"
+
+#define HARP_MAX_STAGES 24
+
+// Stage geometry handed to kernels by value.
+struct StageTable {
+    int32_t m;
+    int32_t b[HARP_MAX_STAGES];       // radix b_t
+    int32_t s[HARP_MAX_STAGES];       // stride s_t = prod_{j<t} b_j
+    int64_t off[HARP_MAX_STAGES];     // offset (in floats) of stage t in the block array
+};
+
+struct FastPlan;   // tensor-core path data (harp_fast.cu)
+
+struct harp_plan {
+    int64_t d = 0;
+    int device = 0;
+    StageTable st{};
+    int64_t n_params = 0;
+    float *d_blocks = nullptr;        // [sum_t d*b_t] fp32, stage after stage
+    int32_t *d_perm = nullptr;        // nullptr = identity
+    int8_t *d_signs = nullptr;        // nullptr = all +1
+    // host copies (used to derive kernel-specific layouts)
+    std::vector<int32_t> h_perm;
+    std::vector<int8_t> h_signs;
+    std::vector<float> h_blocks;
+    FastPlan *fast = nullptr;
+    // staging owned by harp_apply_host
+    void *stage_buf[2] = {nullptr, nullptr};
+    int64_t stage_bytes = 0;
+    cudaStream_t stage_stream[2] = {nullptr, nullptr};
+};
+
+extern std::atomic<int64_t> g_harp_launches;
+
+// generic CUDA-core path (harp_generic.cu)
+harp_status_t harp_generic_supported(const harp_plan *plan, harp_dtype_t dtype);
+harp_status_t harp_generic_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype,
+                                 int transpose, cudaStream_t stream);
+
+// tensor-core path (harp_fast.cu)
+harp_status_t harp_fast_build(harp_plan *plan);     // HARP_OK or HARP_ERR_UNSUPPORTED (plan->fast stays null)
+void harp_fast_destroy(harp_plan *plan);
+harp_status_t harp_fast_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype,
+                              int transpose, cudaStream_t stream);
+
+// out-of-place matrix transpose, rows x cols -> cols x rows (harp_two_sided.cu)
+harp_status_t harp_transpose_matrix(const void *src, void *dst, int64_t rows, int64_t cols,
+                                    harp_dtype_t dtype, cudaStream_t stream);
+
+static inline size_t harp_dtype_size(harp_dtype_t t) { return t == HARP_F32 ? 4 : 2; }

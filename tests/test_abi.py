@@ -1,0 +1,80 @@
+"""The C-ABI library loads, exports every function include/harp.h declares, and
+rejects bad input before touching CUDA (runs without a GPU)."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import paper_2605_29843_b200 as harp
+from paper_2605_29843_b200 import build as harp_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    harp_build.build()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "harp.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(harp_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    names = declared_functions()
+    assert {"harp_plan_create", "harp_apply", "harp_apply_two_sided", "harp_plan_destroy"} <= set(names)
+    L = harp.lib()
+    for n in names:
+        assert getattr(L, n) is not None, n
+
+
+def test_binding_has_the_same_names():
+    for n in declared_functions():
+        if n in ("harp_plan_destroy", "harp_status_string", "harp_apply_ex"):
+            continue                     # owned by Plan.__del__ / status_string / harp_apply(kernel=)
+        assert hasattr(harp, n), n
+
+
+def _eye_blocks(d, radices):
+    return [np.broadcast_to(np.eye(b, dtype=np.float32), (d // b, b, b)).copy() for b in radices]
+
+
+@pytest.mark.parametrize("kwargs,code", [
+    (dict(d=8, radices=(2, 2, 3)), 3),                 # product != d
+    (dict(d=8, radices=(2, 4, 1)), 3),                 # radix < 2
+    (dict(d=1, radices=(1,)), 2),                      # d < 2
+    (dict(d=8, radices=(2, 2, 2), perm=[0, 1, 2, 3, 4, 5, 6, 6]), 4),
+    (dict(d=8, radices=(2, 2, 2), perm=[0, 1, 2, 3, 4, 5, 6, 8]), 4),
+    (dict(d=8, radices=(2, 2, 2), signs=[1, 1, 1, 0, 1, 1, 1, 1]), 5),
+])
+def test_plan_validation_codes(kwargs, code):
+    d, radices = kwargs["d"], kwargs["radices"]
+    blocks = [np.zeros((max(1, d // max(b, 1)), max(b, 1), max(b, 1)), np.float32) for b in radices]
+    st, plan = harp.harp_plan_create_status(d, radices, kwargs.get("perm"), kwargs.get("signs"), blocks)
+    assert st == code and plan is None
+    assert isinstance(harp.status_string(st), str) and harp.status_string(st) != "ok"
+
+
+def test_null_arguments():
+    L = harp.lib()
+    assert L.harp_apply(None, None, 4, 0, 0, None) == 1
+    assert L.harp_apply_two_sided(None, 0, None, None, None, None) == 1
+    assert L.harp_plan_dim(None) == -1
+    assert L.harp_two_sided_scratch_bytes(None, None, 0) == 0
+    out = ctypes.c_void_p()
+    assert L.harp_plan_create(ctypes.byref(out), 8, 3, None, None, None, None) == 1
+    L.harp_plan_destroy(None)
+    assert harp.status_string(0) == "ok"
+    assert harp.harp_launch_count() >= 0
+
+
+def test_no_gpu_means_an_error_not_a_fallback():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    st, plan = harp.harp_plan_create_status(8, (2, 2, 2), None, None, _eye_blocks(8, (2, 2, 2)))
+    assert st in (9, 10) and plan is None

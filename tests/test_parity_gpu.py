@@ -1,0 +1,202 @@
+"""GPU parity: libharp.so (through the C ABI) against the CPU oracle, element by
+element on the same seeded inputs.  Metric: max_i |got_i - want_i| / ||want||_2 per
+row, maximised over rows; 1e-5 for fp32 I/O, 8e-3 for bf16 I/O."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2605_29843_b200 as harp
+from oracle import c_oracle, harp_oracle as orc
+from paper_2605_29843_b200 import workloads as wl
+from harp_testlib import TOL, gpu_apply, host_rows, promote, to_device, to_host_f64
+
+pytestmark = pytest.mark.gpu
+
+KERNELS = [harp.KERNEL_GENERIC, harp.KERNEL_AUTO]
+
+TINY = [(2, 2, 2), (4, 4), (2, 3), (7, 2), (3, 5, 2), (16, 4), (43,), (2, 2, 7), (8, 8), (5, 4, 3),
+        (16, 16, 8), (2, 43), (8, 7, 2), (4, 4, 4, 4), (2,) * 9, (16, 8, 7), (3, 3, 3, 3)]
+
+
+@pytest.mark.parametrize("radices", TINY)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_tiny_schedules_forward_and_transpose(radices, dtype, kernel):
+    spec = wl.tiny_plan(31, radices, kind="qr", perm="random", signs=True)
+    oplan = orc.OraclePlan.from_spec(spec)
+    plan = harp.plan_from_spec(spec)
+    rng = np.random.default_rng(5)
+    for n_rows in (1, 2, 7, 33):
+        xh = host_rows(rng.standard_normal((n_rows, spec.d)), dtype)
+        x64 = promote(xh, dtype)
+        got, guards = gpu_apply(plan, xh, dtype, False, kernel)
+        assert guards
+        assert orc.rel_err_rows(got, orc.forward(oplan, x64)) <= TOL[dtype]
+        got, guards = gpu_apply(plan, xh, dtype, True, kernel)
+        assert guards
+        assert orc.rel_err_rows(got, orc.transpose(oplan, x64)) <= TOL[dtype]
+
+
+@pytest.mark.parametrize("radices", [(2, 2, 2), (3, 5, 2), (4,) * 6, (16, 16, 8, 7), (2,) * 8 + (43,)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_identity_blocks_are_a_bit_exact_sign_and_gather(radices, dtype, kernel):
+    spec = wl.tiny_plan(17, radices, kind="identity", perm="random", signs=True)
+    plan = harp.plan_from_spec(spec)
+    rng = np.random.default_rng(6)
+    xh = host_rows(rng.standard_normal((9, spec.d)), dtype)
+    x64 = promote(xh, dtype)
+    got, guards = gpu_apply(plan, xh, dtype, False, kernel)
+    assert guards and np.array_equal(got, (x64 * spec.signs)[:, spec.perm])
+    back, guards = gpu_apply(plan, host_rows(got, dtype), dtype, True, kernel)
+    assert guards and np.array_equal(back, x64)
+
+
+CFG_ROWS = {1: 300, 2: 300, 3: 131, 4: 100, 5: 67}
+
+
+def _cfg_plan_and_data(cfg, n_rows):
+    w = wl.config(cfg, n_rows=n_rows)
+    spec = w.plans["in"] if cfg == 5 else w.plans["q"]
+    data = w.data["x"]
+    return w, spec, data
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_configs_reduced_rows_all_elements(cfg, kernel):
+    n = CFG_ROWS[cfg]
+    w, spec, data = _cfg_plan_and_data(cfg, n)
+    plan = harp.plan_from_spec(spec)
+    cplan = c_oracle.CPlan(spec)
+    xh = data.rows(0, n)
+    x64 = data.rows_f64(0, n)
+    got, guards = gpu_apply(plan, xh, data.dtype, False, kernel)
+    want = c_oracle.forward(cplan, x64)
+    assert guards
+    assert orc.rel_err_rows(got, want) <= w.tol
+    got_t, guards = gpu_apply(plan, xh, data.dtype, True, kernel)
+    assert guards
+    assert orc.rel_err_rows(got_t, c_oracle.transpose(cplan, x64)) <= w.tol
+    # forward then transpose returns the input up to two roundings
+    back, _ = gpu_apply(plan, host_rows(got, data.dtype), data.dtype, True, kernel)
+    assert orc.rel_err_rows(back, x64) <= 2 * w.tol
+
+
+@pytest.mark.parametrize("cfg", [4])
+def test_decode_batches(cfg):
+    w, spec, data = _cfg_plan_and_data(cfg, 16)
+    plan = harp.plan_from_spec(spec)
+    cplan = c_oracle.CPlan(spec)
+    for n in w.extra["decode_rows"]:
+        got, guards = gpu_apply(plan, data.rows(0, n), data.dtype)
+        assert guards
+        assert orc.rel_err_rows(got, c_oracle.forward(cplan, data.rows_f64(0, n))) <= w.tol
+
+
+def _upload_rows(data, n_rows, chunk=4096):
+    tdt = torch.float32 if data.dtype == "f32" else torch.bfloat16
+    x = torch.empty((n_rows, data.d), dtype=tdt, device="cuda")
+    for r in range(0, n_rows, chunk):
+        k = min(chunk, n_rows - r)
+        x[r:r + k] = to_device(data.rows(r, k), data.dtype)
+    return x
+
+
+@pytest.mark.parametrize("cfg", [1, 2, 3, 4, 5])
+def test_full_size_sampled_rows(cfg):
+    """Full row count in the launch configuration the benchmark times; rows sampled
+    across the batch (first, last, tile boundaries, random) are checked in full."""
+    w, spec, data = _cfg_plan_and_data(cfg, None)
+    n = data.n_rows
+    plan = harp.plan_from_spec(spec)
+    cplan = c_oracle.CPlan(spec)
+    x = _upload_rows(data, n)
+    rng = np.random.default_rng(cfg)
+    rows = sorted(set([0, 1, 15, 16, 17, n // 2, n - 17, n - 2, n - 1] + rng.integers(0, n, 23).tolist()))
+    harp.apply_(plan, x)
+    torch.cuda.synchronize()
+    got = to_host_f64(x[rows])
+    want = c_oracle.forward(cplan, np.concatenate([data.rows_f64(r, 1) for r in rows]))
+    assert orc.rel_err_rows(got, want) <= w.tol
+    # norm preservation holds for every row at any size
+    nrm = torch.linalg.vector_norm(x.float(), dim=1).double().cpu().numpy()
+    want_nrm = np.linalg.norm(want, axis=1)
+    assert np.allclose(nrm[rows], want_nrm, rtol=5e-3)
+    harp.apply_(plan, x, transpose=True)
+    torch.cuda.synchronize()
+    back = to_host_f64(x[rows])
+    orig = np.concatenate([data.rows_f64(r, 1) for r in rows])
+    assert orc.rel_err_rows(back, orig) <= 2 * w.tol
+
+
+def test_two_sided_tiny_against_dense():
+    for dtype in ("f32", "bf16"):
+        p_out = wl.tiny_plan(41, (3, 4, 2), perm="random")
+        p_in = wl.tiny_plan(42, (2, 5, 2, 3), perm="random")
+        po, pi = orc.OraclePlan.from_spec(p_out), orc.OraclePlan.from_spec(p_in)
+        rng = np.random.default_rng(7)
+        wh = host_rows(rng.standard_normal((p_out.d, p_in.d)), dtype)
+        w64 = promote(wh, dtype)
+        wd = to_device(wh, dtype)
+        harp.two_sided_(wd, harp.plan_from_spec(p_out), harp.plan_from_spec(p_in))
+        torch.cuda.synchronize()
+        want = orc.dense(po).T @ w64 @ orc.dense(pi)
+        got = to_host_f64(wd)
+        assert np.max(np.abs(got - want)) / np.linalg.norm(want, axis=1).min() <= TOL[dtype] * 2
+        assert np.allclose(want, orc.two_sided(po, pi, w64), atol=1e-12)
+
+
+def test_two_sided_full_size():
+    w = wl.config(5)
+    p_out, p_in, wdata = w.plans["out"], w.plans["in"], w.data["w"]
+    W = _upload_rows(wdata, wdata.n_rows)
+    W0 = W.clone()
+    plan_out, plan_in = harp.plan_from_spec(p_out), harp.plan_from_spec(p_in)
+    scratch = torch.empty(harp.harp_two_sided_scratch_bytes(plan_out, plan_in, harp.HARP_BF16),
+                          dtype=torch.uint8, device="cuda")
+    harp.two_sided_(W, plan_out, plan_in, scratch)
+    torch.cuda.synchronize()
+    # Frobenius norm is preserved
+    n0 = torch.linalg.vector_norm(W0.float()).item()
+    n1 = torch.linalg.vector_norm(W.float()).item()
+    assert abs(n1 - n0) / n0 < 2e-3
+    # full element-wise comparison with the oracle
+    want = c_oracle.two_sided(c_oracle.CPlan(p_out), c_oracle.CPlan(p_in), wdata.rows_f64(0, wdata.n_rows))
+    got = to_host_f64(W)
+    # tolerance relative to the norm of the row (row side) and of the column (column side)
+    err = np.abs(got - want)
+    row_n = np.linalg.norm(want, axis=1, keepdims=True)
+    col_n = np.linalg.norm(want, axis=0, keepdims=True)
+    assert np.max(err / np.minimum(row_n, col_n)) <= 2 * w.tol
+    # the layer function is unchanged: y = x W^T = transpose_out(forward_in(x) W~^T)
+    x = np.random.default_rng(3).standard_normal((2, p_in.d))
+    w0 = to_host_f64(W0)
+    y = c_oracle.transpose(c_oracle.CPlan(p_out), c_oracle.forward(c_oracle.CPlan(p_in), x) @ got.T)
+    ref = x @ w0.T
+    assert np.max(np.abs(y - ref)) / np.linalg.norm(ref, axis=1).min() < 2e-2
+
+
+def test_host_buffer_entry_point():
+    w, spec, data = _cfg_plan_and_data(2, 600)
+    plan = harp.plan_from_spec(spec)
+    xh = torch.from_numpy(data.rows(0, 600).view(np.int16)).view(torch.bfloat16).pin_memory()
+    harp.harp_apply_host(plan, xh.data_ptr(), 600, harp.HARP_BF16, False)
+    want = c_oracle.forward(c_oracle.CPlan(spec), data.rows_f64(0, 600))
+    assert orc.rel_err_rows(to_host_f64(xh), want) <= w.tol
+
+
+def test_status_codes_on_device():
+    spec = wl.tiny_plan(1, (2, 2, 2))
+    plan = harp.plan_from_spec(spec)
+    assert harp.harp_plan_dim(plan) == 8
+    L = harp.lib()
+    x = torch.zeros((4, 8), device="cuda")
+    assert L.harp_apply(plan.handle, x.data_ptr(), 0, 0, 0, None) == 0          # empty batch
+    assert L.harp_apply(plan.handle, None, 4, 0, 0, None) == 1
+    assert L.harp_apply(plan.handle, x.data_ptr(), -1, 0, 0, None) == 2
+    assert L.harp_apply(plan.handle, x.data_ptr(), 4, 7, 0, None) == 6
+    before = harp.harp_launch_count()
+    harp.apply_(plan, x)
+    torch.cuda.synchronize()
+    assert harp.harp_launch_count() > before
