@@ -1,0 +1,362 @@
+#!/usr/bin/env python
+"""Benchmark of the HARP apply hot path on B200.
+
+One step = one pass of the apply path over one synthetic batch of the headline
+workload (d = 4096 = 4^6, radix-4 schedule, sign diagonal, base-4 digit-reversal
+permutation, 16384 bf16 rows): a forward apply (y = x Q) of the batch followed by a
+transpose apply (x = y Q^T) of a batch.  `value` counts row-applies per second
+(2 * n_rows per step), whole job.  Four device buffers (134 MB each) are rotated so a
+buffer is touched again only after three others (> 3x the 126 MB L2) have streamed by.
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
+`--all-configs` adds per-configuration measurements under the key "per_config".
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2605_29843_b200 import workloads as wl  # noqa: E402
+
+METRIC = "harp_apply_rows_per_s"
+UNIT = "rows/s"
+WORKLOAD = "cfg2: d=4096 radix-4 x6, signs + digit-reversal perm, 16384 rows bf16, forward+transpose per step"
+N_BUF = 4
+# DRAM bytes (read+write) per launch of the dominant kernel on the headline workload,
+# from the ncu capture summarised in profiles/ (None until captured).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return float(j["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons in the background."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int, period_ms: int = 50):
+        self.samples = []
+        self.proc = None
+        self.t0 = self.t1 = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-i", str(index), "-lms", str(period_ms)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL,
+                text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def mark_start(self):
+        self.t0 = time.time()
+
+    def mark_end(self):
+        self.t1 = time.time()
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        time.sleep(0.06)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        inside = [s for t, s in self.samples if self.t0 is not None and self.t0 - 0.05 <= t <= self.t1 + 0.1]
+        use = inside if inside else [s for _, s in self.samples]
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in use:
+            f = [v.strip() for v in s.split(",")]
+            try:
+                sm.append(float(f[0]))
+                smax.append(float(f[1]))
+            except Exception:
+                continue
+            for name, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "reasons": sorted(reasons), "samples": len(use)}
+
+
+# ------------------------------------------------------------------ reference arm
+
+def oracle_step(cplan, x64, c_oracle):
+    c_oracle.forward(cplan, x64)
+    c_oracle.transpose(cplan, x64)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import c_oracle
+    w = wl.config(2)
+    spec, data = w.plans["q"], w.data["x"]
+    cplan = c_oracle.CPlan(spec)
+    sample_rows = args.ref_rows
+    x64 = data.rows_f64(0, sample_rows)
+    for _ in range(max(1, min(args.warmup, 2))):
+        oracle_step(cplan, x64, c_oracle)
+    steps = max(1, min(args.steps, 20))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_step(cplan, x64, c_oracle)
+    dt = time.perf_counter() - t0
+    val = 2 * sample_rows * steps / dt
+    sample = f"{sample_rows} of {data.n_rows} rows per step, forward+transpose, {steps} steps"
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": sample},
+            "cpu_baseline": {"value": val, "unit": UNIT, "cores": c_oracle.threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------ GPU arm
+
+def cpu_baseline(spec, data):
+    from oracle import c_oracle
+    cplan = c_oracle.CPlan(spec)
+    probe = 256
+    x64 = data.rows_f64(0, probe)
+    t0 = time.perf_counter()
+    oracle_step(cplan, x64, c_oracle)
+    dt = time.perf_counter() - t0
+    rows = int(min(data.n_rows, max(probe, probe * 12.0 / max(dt, 1e-6))))
+    rows = (rows // 256) * 256 or 256
+    x64 = data.rows_f64(0, rows)
+    t0 = time.perf_counter()
+    oracle_step(cplan, x64, c_oracle)
+    one = time.perf_counter() - t0
+    reps = int(max(1, min(20, round(10.0 / max(one, 1e-3)))))
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        oracle_step(cplan, x64, c_oracle)
+    dt = time.perf_counter() - t0
+    return {"value": 2 * rows * reps / dt, "unit": UNIT, "cores": c_oracle.threads(), "kind": "oracle",
+            "sample": f"first {rows} of {data.n_rows} rows, forward+transpose, {reps} passes, {dt:.1f} s"}
+
+
+def time_region(torch, fn, iters):
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for i in range(iters):
+        fn(i)
+    end.record()
+    end.synchronize()
+    return start.elapsed_time(end) * 1e-3
+
+
+def bench_extra_configs(torch, harp, kernel, peak):
+    """Per-configuration apply throughput (forward and transpose), decode latency and
+    two-sided time.  Inputs are seeded device-side normals of the configuration's shape
+    (throughput does not depend on the values; parity is covered by the tests)."""
+    out = {}
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(1234)
+    for cfg in (1, 2, 3, 4, 5):
+        w = wl.config(cfg)
+        spec = w.plans["in"] if cfg == 5 else w.plans["q"]
+        data = w.data["x"]
+        plan = harp.plan_from_spec(spec)
+        tdt = torch.float32 if data.dtype == "f32" else torch.bfloat16
+        es = 4 if data.dtype == "f32" else 2
+        nbytes = data.n_rows * data.d * es
+        nbuf = max(2, int(np.ceil(3 * 126e6 / nbytes)) + 1)
+        bufs = [torch.randn((data.n_rows, data.d), generator=gen, device="cuda", dtype=torch.float32).to(tdt)
+                for _ in range(nbuf)]
+        res = {}
+        for name, tr in (("forward", False), ("transpose", True)):
+            for i in range(3):
+                harp.apply_(plan, bufs[i % nbuf], transpose=tr, kernel=kernel)
+            torch.cuda.synchronize()
+            iters = max(5, min(200, int(0.3 / (2 * nbytes / (peak * 1e9) * 3))))
+            dt = time_region(torch, lambda i: harp.apply_(plan, bufs[i % nbuf], transpose=tr, kernel=kernel), iters)
+            gbs = 2 * nbytes * iters / dt / 1e9
+            res[name] = {"rows_per_s": data.n_rows * iters / dt, "GBps": gbs, "frac_of_measured_peak": gbs / peak,
+                         "frac_of_8TBps": gbs / 8000.0, "us_per_launch": 1e6 * dt / iters}
+        if cfg == 4:
+            dec = {}
+            for n in w.extra["decode_rows"]:
+                x = bufs[0][:n]
+                for _ in range(5):
+                    harp.apply_(plan, x, kernel=kernel)
+                torch.cuda.synchronize()
+                dt = time_region(torch, lambda i: harp.apply_(plan, x, kernel=kernel), 200)
+                dec[str(n)] = {"us_per_call": 1e6 * dt / 200}
+            res["decode"] = dec
+        if cfg == 5:
+            del bufs
+            wd = w.data["w"]
+            p_out = harp.plan_from_spec(w.plans["out"])
+            W = (torch.randn((wd.n_rows, wd.d), generator=gen, device="cuda") * 0.02).to(torch.bfloat16)
+            scratch = torch.empty(harp.harp_two_sided_scratch_bytes(p_out, plan, harp.HARP_BF16), dtype=torch.uint8,
+                                  device="cuda")
+            for _ in range(2):
+                harp.two_sided_(W, p_out, plan, scratch)
+            torch.cuda.synchronize()
+            dt = time_region(torch, lambda i: harp.two_sided_(W, p_out, plan, scratch), 10)
+            wbytes = 2 * wd.n_rows * wd.d * 2
+            res["two_sided"] = {"ms": 1e3 * dt / 10, "GBps_vs_1R1W": wbytes * 10 / dt / 1e9,
+                                "frac_of_measured_peak_vs_1R1W": wbytes * 10 / dt / 1e9 / peak}
+        out[w.name] = res
+        bufs = None
+        torch.cuda.empty_cache()
+    return out
+
+
+def run_gpu(args):
+    import torch
+    import torch.distributed as dist
+    import paper_2605_29843_b200 as harp
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the HARP library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    harp.lib()
+    kernel = {"auto": harp.KERNEL_AUTO, "generic": harp.KERNEL_GENERIC, "fast": harp.KERNEL_FAST}[args.kernel]
+
+    w = wl.config(2)
+    spec, data = w.plans["q"], w.data["x"]
+    n_rows, d = data.n_rows, data.d
+    plan = harp.plan_from_spec(spec)
+    # every rank works on a batch of the same shape (weak scaling); rank r draws its own rows
+    host_bits = wl.DataSpec(n_rows, d, "bf16", "normal", seed=data.seed + 1000 * rank).rows(0, n_rows)
+    host = torch.from_numpy(host_bits.view(np.int16)).view(torch.bfloat16)
+    bufs = [host.cuda().clone() for _ in range(N_BUF)]
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        harp.apply_(plan, bufs[(2 * i) % N_BUF], transpose=False, kernel=kernel)
+        harp.apply_(plan, bufs[(2 * i + 1) % N_BUF], transpose=True, kernel=kernel)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    for i in range(max(3, args.warmup)):
+        step(i)
+    barrier()
+    launches0 = harp.harp_launch_count()
+    if sampler:
+        sampler.mark_start()
+    dt = time_region(torch, step, args.steps)
+    barrier()
+    if sampler:
+        sampler.mark_end()
+    launches = harp.harp_launch_count() - launches0
+    t = torch.tensor([dt], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dt_max = float(t.item())
+    clocks = sampler.stop() if sampler else None
+
+    # end to end through the host-buffer entry point: pinned host rows in, results back
+    pinned = [host.clone().pin_memory() for _ in range(2)]
+    e2e_steps = max(2, min(args.steps, 10))
+
+    def e2e_step(i):
+        harp.harp_apply_host(plan, pinned[0].data_ptr(), n_rows, harp.HARP_BF16, False)
+        harp.harp_apply_host(plan, pinned[1].data_ptr(), n_rows, harp.HARP_BF16, True)
+
+    e2e_step(0)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        e2e_step(i)
+    torch.cuda.synchronize()
+    e2e_dt = time.perf_counter() - t0
+    te = torch.tensor([e2e_dt], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e_dt = float(te.item())
+
+    if rank == 0:
+        peak, peak_kind = measured_peaks()
+        row_bytes = d * 2 * 2                                     # bf16 read + write
+        per_launch_s = dt_max / (2 * args.steps)
+        achieved = n_rows * row_bytes / per_launch_s / 1e9
+        line = {
+            "metric": METRIC, "value": world * 2 * n_rows * args.steps / dt_max, "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+            "ms_per_step": 1e3 * dt_max / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16 I/O, fp32 accumulate", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "n_rows": n_rows, "d": d, "kernel": args.kernel,
+                       "l2": f"{N_BUF} rotating 134 MB buffers (inputs larger than L2)", "parallelism": f"rows x{world}"},
+            "clocks": clocks,
+            "e2e": {"value": world * 2 * n_rows * e2e_steps / e2e_dt, "unit": UNIT,
+                    "h2d_bytes_per_step": 2 * n_rows * d * 2, "d2h_bytes_per_step": 2 * n_rows * d * 2,
+                    "api": "harp_apply_host (pinned host rows, chunked copy/compute overlap)"},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBps": achieved / 8000.0,
+                         "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                         "algorithmic_bytes_per_launch": n_rows * row_bytes,
+                         "us_per_launch": 1e6 * per_launch_s},
+        }
+        if not args.no_cpu and world == 1:
+            line["cpu_baseline"] = cpu_baseline(spec, data)
+        if args.all_configs and world == 1:
+            del bufs
+            torch.cuda.empty_cache()
+            line["per_config"] = bench_extra_configs(torch, harp, kernel, peak)
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="harp", choices=["harp", "reference"])
+    ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "fast"])
+    ap.add_argument("--all-configs", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU-oracle baseline")
+    ap.add_argument("--ref-rows", type=int, default=2048)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()
