@@ -105,6 +105,30 @@ harp_status_t harp_apply_two_sided(void *W, harp_dtype_t dtype, const harp_plan_
 int64_t harp_two_sided_scratch_bytes(const harp_plan_t *plan_out, const harp_plan_t *plan_in,
                                      harp_dtype_t dtype);
 
+/* Two-sided processing without any allocation (the paper has no counterpart: this entry
+ * point exists for deployment, not for the method).  It is meant for callers that cannot
+ * allocate device memory at call time -- a serving process whose memory pool was sized
+ * once at start-up, a host framework that owns the whole device budget, or any context in
+ * which an allocation would synchronise or fail.  It computes exactly what
+ * harp_apply_two_sided computes, but keeps the transposed copy of W in a fixed array that
+ * is compiled into the library; every device that loads the library holds that array
+ * (harp_two_sided_static_capacity_bytes() = 32 MiB) until the process exits.
+ *   W        DEVICE d_out x d_in row-major, overwritten; d_out*d_in*sizeof(dtype) must not
+ *            exceed the capacity, otherwise HARP_ERR_TOO_LARGE and nothing is launched
+ *   plans    must live on the current device (else HARP_ERR_DIM_MISMATCH)
+ * No cudaMalloc/cudaFree or other allocating call is made.  The first call on a device
+ * looks up the array's device address; make that first call outside any stream capture.
+ * All calls share the one array, which keeps whatever the last call left in it (nothing
+ * needs to start at zero: every byte is written before it is read).  Two calls that
+ * overlap on the GPU -- different streams, or different host threads -- race on it; run
+ * them one after the other.  Asynchronous on stream. */
+harp_status_t harp_apply_two_sided_static(void *W, harp_dtype_t dtype,
+                                          const harp_plan_t *plan_out,
+                                          const harp_plan_t *plan_in, void *stream);
+
+/* Capacity in bytes of the fixed scratch array used by harp_apply_two_sided_static. */
+int64_t harp_two_sided_static_capacity_bytes(void);
+
 /* Apply to rows that live in HOST memory (pinned memory gives full copy speed):
  * copies chunks host->device, applies, copies back, on two internal streams so that
  * copies overlap kernels; returns after the last copy has completed.  The device staging

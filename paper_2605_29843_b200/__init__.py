@@ -51,6 +51,10 @@ def lib() -> ctypes.CDLL:
         L.harp_apply_two_sided.argtypes = [vp, ctypes.c_int, vp, vp, vp, vp]
         L.harp_two_sided_scratch_bytes.restype = i64
         L.harp_two_sided_scratch_bytes.argtypes = [vp, vp, ctypes.c_int]
+        L.harp_apply_two_sided_static.restype = ctypes.c_int
+        L.harp_apply_two_sided_static.argtypes = [vp, ctypes.c_int, vp, vp, vp]
+        L.harp_two_sided_static_capacity_bytes.restype = i64
+        L.harp_two_sided_static_capacity_bytes.argtypes = []
         L.harp_apply_host.restype = ctypes.c_int
         L.harp_apply_host.argtypes = [vp, vp, i64, ctypes.c_int, ctypes.c_int]
         L.harp_launch_count.restype = i64
@@ -133,6 +137,20 @@ def harp_apply_two_sided(w_ptr: int, dtype: int, plan_out: Plan, plan_in: Plan,
                                     scratch_ptr or None, stream or None)
     if st != HARP_OK:
         raise HarpError(st, "harp_apply_two_sided")
+
+
+def harp_apply_two_sided_static(w_ptr: int, dtype: int, plan_out: Plan, plan_in: Plan, stream: int = 0) -> int:
+    """Two-sided processing for callers that cannot allocate device memory (fixed memory
+    pools, device budgets owned by another framework): the transposed copy of W lives in a
+    32 MiB array inside the library instead of a buffer obtained at call time.  Returns the
+    status code (0 = ok, 11 = W larger than the fixed capacity) instead of raising, so a
+    caller can fall back to ``harp_apply_two_sided`` with its own scratch."""
+    return int(lib().harp_apply_two_sided_static(w_ptr, int(dtype), plan_out.handle, plan_in.handle,
+                                                 stream or None))
+
+
+def harp_two_sided_static_capacity_bytes() -> int:
+    return int(lib().harp_two_sided_static_capacity_bytes())
 
 
 def harp_two_sided_scratch_bytes(plan_out: Plan, plan_in: Plan, dtype: int) -> int:
