@@ -1,9 +1,685 @@
-// Tensor-core path (placeholder until the kernels land): reports "unsupported" so that
-// dispatch uses the generic kernel.
+// Tensor-core path for bf16 rows (sm_100a).
+//
+// Plan time: adjacent stages are fused into "phases" whose dense block has size
+// B in {8, 16} (two radix-4 stages -> one 16x16 block, four radix-2 stages -> 16x16, one
+// radix-8 stage -> 8x8, ...).  A fused block is the product of its stages' kernels on the B
+// coordinates it touches, computed in fp64 and rounded once to bf16; the sign diagonal is
+// folded into the first phase.  Per phase the blocks are stored in the register layout of
+// mma.sync (one 16-byte load per lane and block).
+//
+// Run time: a CTA keeps a tile of 16 whole rows in shared memory as bf16 (one HBM read and
+// one HBM write per row) and runs the phases on it.  A phase is a batch of tiny GEMMs
+// out[16 rows x B] = in[16 rows x B] . F_c[B x B] (fp32 accumulate), one per block c, with
+// the 16 rows as the M dimension of mma.sync.m16n8k16.  Coordinates of a block that are
+// not adjacent in memory are fetched for eight neighbouring blocks at once with 16-byte
+// loads and re-paired with byte permutes, so that shared memory is only touched with
+// 16-byte, bank-conflict-free accesses; every thread writes exactly the locations it
+// read, so a phase needs no barrier between its loads and stores.
+//
+// Permutations: identity, or any permutation that maps every aligned run of eight source
+// coordinates onto the same slot of eight different first-phase blocks (mixed-radix digit
+// reversal is of this kind).  For those the first phase reads its operands straight from
+// global memory (forward) or the last phase writes straight to global memory (transpose),
+// so the permutation costs no extra pass.  Other permutations use the generic kernel.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <map>
+#include <new>
+
 #include "harp_internal.h"
 
-harp_status_t harp_fast_build(harp_plan *plan) { (void)plan; return HARP_ERR_UNSUPPORTED; }
-void harp_fast_destroy(harp_plan *plan) { (void)plan; }
-harp_status_t harp_fast_apply(const harp_plan *, void *, int64_t, harp_dtype_t, int, cudaStream_t) {
-    return HARP_ERR_UNSUPPORTED;
+namespace {
+
+constexpr int kMaxPhases = 8;
+constexpr int kTileRows = 16;
+constexpr int kThreads = 512;
+constexpr int kWarps = kThreads / 32;
+
+enum PhaseMode : int32_t {
+    MODE_CC = 0,   // contiguous block in shared memory, in place (ldmatrix / stmatrix)
+    MODE_SS = 1,   // strided block in shared memory, eight blocks per item, in place
+    MODE_GS = 2,   // operands gathered from global memory, result to contiguous smem blocks
+    MODE_CG = 3    // operands from contiguous smem blocks, result scattered to global memory
+};
+
+struct PhaseDesc {
+    const uint4 *bfrag;        // [item][block in item][lane] fragments
+    const int32_t *items;      // per-item table (layout depends on mode)
+    int32_t n_items;
+    int32_t mode;
+    int32_t B;                 // 8 or 16
+    int32_t lane_step;         // element offset between the slots of lanes q and q+1
+    int32_t j_off[4];          // element offsets of a lane's slots
+};
+
+struct FastParams {
+    int32_t n_phases;
+    int32_t d;
+    int32_t pitch;             // elements per shared-memory row
+    int32_t copy_in;           // load the tile with cp.async before the first phase
+    int32_t copy_out;          // store the tile from shared memory after the last phase
+    const int32_t *chunk_phys; // [d/8] shared-memory element offset of every 8-coordinate chunk
+    PhaseDesc ph[kMaxPhases];
+};
+
+// ----------------------------------------------------------------------------- device
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void sts128(uint32_t addr, const uint4 &v) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ uint4 ldg128_stream(const void *p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void stg128(void *p, const uint4 &v) {
+    asm volatile("st.global.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void stmatrix_x4(uint32_t addr, uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3) {
+    asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(r0), "r"(r1), "r"(r2), "r"(r3) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x2(uint32_t (&r)[2], uint32_t addr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x2.shared.b16 {%0,%1}, [%2];" : "=r"(r[0]), "=r"(r[1]) : "r"(addr));
+}
+__device__ __forceinline__ void stmatrix_x2(uint32_t addr, uint32_t r0, uint32_t r1) {
+    asm volatile("stmatrix.sync.aligned.m8n8.x2.shared.b16 [%0], {%1,%2};" ::"r"(addr), "r"(r0), "r"(r1) : "memory");
+}
+// D(16x8, fp32) = A(16x16, bf16) . B(16x8, bf16)
+__device__ __forceinline__ void mma_k16(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%10,%10,%10};"
+        : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
+}
+// D(16x8, fp32) = A(16x8, bf16) . B(8x8, bf16)
+__device__ __forceinline__ void mma_k8(float (&c)[4], const uint32_t (&a)[2], uint32_t b0) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%7,%7,%7,%7};"
+        : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(b0), "f"(0.f));
+}
+// {lo, hi} -> packed bf16x2, round to nearest even
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+__device__ __forceinline__ uint32_t pair_lo(uint32_t x, uint32_t y) { return __byte_perm(x, y, 0x5410); }
+__device__ __forceinline__ uint32_t pair_hi(uint32_t x, uint32_t y) { return __byte_perm(x, y, 0x7632); }
+__device__ __forceinline__ uint32_t word_of(const uint4 &v, int w) {
+    return w == 0 ? v.x : (w == 1 ? v.y : (w == 2 ? v.z : v.w));
+}
+__device__ __forceinline__ void set_word(uint4 &v, int w, uint32_t x) {
+    if (w == 0) v.x = x; else if (w == 1) v.y = x; else if (w == 2) v.z = x; else v.w = x;
+}
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
+// Eight blocks at once: raw[j][h] holds, for slot j of this lane and row half h, the values
+// of the eight neighbouring blocks.  Computes the eight block products and leaves the
+// results in raw (same slots, same rows) -- B = 16.
+template <bool CONTIG_OUT>
+__device__ __forceinline__ void octet_mma16(uint4 (&raw)[4][2], const uint4 *bptr, uint32_t (&mats)[8][4]) {
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        float acc[2][2][4];
+#pragma unroll
+        for (int ee = 0; ee < 2; ++ee) {
+            const uint4 bf = __ldg(bptr + (2 * w + ee) * 32);
+            uint32_t a[4];
+            if (ee == 0) {
+                a[0] = pair_lo(word_of(raw[0][0], w), word_of(raw[1][0], w));
+                a[1] = pair_lo(word_of(raw[0][1], w), word_of(raw[1][1], w));
+                a[2] = pair_lo(word_of(raw[2][0], w), word_of(raw[3][0], w));
+                a[3] = pair_lo(word_of(raw[2][1], w), word_of(raw[3][1], w));
+            } else {
+                a[0] = pair_hi(word_of(raw[0][0], w), word_of(raw[1][0], w));
+                a[1] = pair_hi(word_of(raw[0][1], w), word_of(raw[1][1], w));
+                a[2] = pair_hi(word_of(raw[2][0], w), word_of(raw[3][0], w));
+                a[3] = pair_hi(word_of(raw[2][1], w), word_of(raw[3][1], w));
+            }
+            mma_k16(acc[ee][0], a, bf.x, bf.y);
+            mma_k16(acc[ee][1], a, bf.z, bf.w);
+        }
+        if (CONTIG_OUT) {
+#pragma unroll
+            for (int ee = 0; ee < 2; ++ee) {
+                mats[2 * w + ee][0] = pack_bf16(acc[ee][0][0], acc[ee][0][1]);
+                mats[2 * w + ee][1] = pack_bf16(acc[ee][0][2], acc[ee][0][3]);
+                mats[2 * w + ee][2] = pack_bf16(acc[ee][1][0], acc[ee][1][1]);
+                mats[2 * w + ee][3] = pack_bf16(acc[ee][1][2], acc[ee][1][3]);
+            }
+        } else {
+#pragma unroll
+            for (int k = 0; k < 2; ++k)
+#pragma unroll
+                for (int i = 0; i < 2; ++i)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        set_word(raw[i + 2 * k][h], w, pack_bf16(acc[0][k][i + 2 * h], acc[1][k][i + 2 * h]));
+        }
+    }
+}
+
+// B = 8: slots j = 0, 1 only.
+__device__ __forceinline__ void octet_mma8(uint4 (&raw)[2][2], const uint32_t *bptr) {
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        float acc[2][4];
+#pragma unroll
+        for (int ee = 0; ee < 2; ++ee) {
+            const uint32_t bf = __ldg(bptr + (2 * w + ee) * 32);
+            uint32_t a[2];
+            if (ee == 0) {
+                a[0] = pair_lo(word_of(raw[0][0], w), word_of(raw[1][0], w));
+                a[1] = pair_lo(word_of(raw[0][1], w), word_of(raw[1][1], w));
+            } else {
+                a[0] = pair_hi(word_of(raw[0][0], w), word_of(raw[1][0], w));
+                a[1] = pair_hi(word_of(raw[0][1], w), word_of(raw[1][1], w));
+            }
+            mma_k8(acc[ee], a, bf);
+        }
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) set_word(raw[i][h], w, pack_bf16(acc[0][i + 2 * h], acc[1][i + 2 * h]));
+    }
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles, FastParams P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const uint32_t sbase = smem_u32(smem_raw);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, q = lane & 3;
+    const int d = P.d, pitch = P.pitch;
+
+    for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        const int64_t row0 = tile * kTileRows;
+        // rows past the end of the batch are computed on a copy of the last row and never stored
+        const int64_t last = n_rows - 1;
+        const int64_t rowA = min(row0 + g, last), rowB = min(row0 + g + 8, last);
+        const bool okA = row0 + g < n_rows, okB = row0 + g + 8 < n_rows;
+        __nv_bfloat16 *xA = x + rowA * d, *xB = x + rowB * d;
+
+        if (P.copy_in) {
+            const int chunks = d >> 3;
+            for (int idx = threadIdx.x; idx < kTileRows * chunks; idx += kThreads) {
+                const int r = idx / chunks, c = idx - r * chunks;
+                const int64_t row = min(row0 + r, last);
+                cp_async16(sbase + 2u * (uint32_t)(r * pitch + __ldg(P.chunk_phys + c)), x + row * d + 8 * c);
+            }
+            cp_async_wait_all();
+            __syncthreads();
+        }
+
+        for (int p = 0; p < P.n_phases; ++p) {
+            const PhaseDesc &ph = P.ph[p];
+            if (ph.mode == MODE_CC) {
+                // lane -> (matrix row, 8-column half) of the 16x16 (or 16x8) operand tile
+                const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
+                if (ph.B == 16) {
+                    for (int it = warp; it < ph.n_items; it += kWarps) {
+                        const uint32_t addr = sbase + 2u * (uint32_t)(mrow * pitch + __ldg(ph.items + it) + mcol);
+                        const uint4 bf = __ldg(ph.bfrag + (size_t)it * 32 + lane);
+                        uint32_t a[4];
+                        ldmatrix_x4(a, addr);
+                        float c0[4], c1[4];
+                        mma_k16(c0, a, bf.x, bf.y);
+                        mma_k16(c1, a, bf.z, bf.w);
+                        stmatrix_x4(addr, pack_bf16(c0[0], c0[1]), pack_bf16(c0[2], c0[3]), pack_bf16(c1[0], c1[1]),
+                                    pack_bf16(c1[2], c1[3]));
+                    }
+                } else {
+                    const uint32_t *bf8 = reinterpret_cast<const uint32_t *>(ph.bfrag);
+                    const int mrow2 = (lane & 15);
+                    for (int it = warp; it < ph.n_items; it += kWarps) {
+                        const uint32_t addr = sbase + 2u * (uint32_t)(mrow2 * pitch + __ldg(ph.items + it));
+                        const uint32_t bf = __ldg(bf8 + (size_t)it * 32 + lane);
+                        uint32_t a[2];
+                        ldmatrix_x2(a, addr);
+                        float c0[4];
+                        mma_k8(c0, a, bf);
+                        stmatrix_x2(addr, pack_bf16(c0[0], c0[1]), pack_bf16(c0[2], c0[3]));
+                    }
+                }
+            } else if (ph.mode == MODE_SS) {
+                const uint32_t rA = sbase + 2u * (uint32_t)(g * pitch + q * ph.lane_step);
+                const uint32_t rB = rA + 2u * (uint32_t)(8 * pitch);
+                if (ph.B == 16) {
+                    for (int it = warp; it < ph.n_items; it += kWarps) {
+                        const uint32_t base = 2u * (uint32_t)__ldg(ph.items + it);
+                        uint4 raw[4][2];
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            raw[j][0] = lds128(rA + base + 2u * ph.j_off[j]);
+                            raw[j][1] = lds128(rB + base + 2u * ph.j_off[j]);
+                        }
+                        uint32_t unused[8][4];
+                        octet_mma16<false>(raw, ph.bfrag + (size_t)it * 256 + lane, unused);
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            sts128(rA + base + 2u * ph.j_off[j], raw[j][0]);
+                            sts128(rB + base + 2u * ph.j_off[j], raw[j][1]);
+                        }
+                    }
+                } else {
+                    const uint32_t *bf8 = reinterpret_cast<const uint32_t *>(ph.bfrag);
+                    for (int it = warp; it < ph.n_items; it += kWarps) {
+                        const uint32_t base = 2u * (uint32_t)__ldg(ph.items + it);
+                        uint4 raw[2][2];
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            raw[j][0] = lds128(rA + base + 2u * ph.j_off[j]);
+                            raw[j][1] = lds128(rB + base + 2u * ph.j_off[j]);
+                        }
+                        octet_mma8(raw, bf8 + (size_t)it * 256 + lane);
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            sts128(rA + base + 2u * ph.j_off[j], raw[j][0]);
+                            sts128(rB + base + 2u * ph.j_off[j], raw[j][1]);
+                        }
+                    }
+                }
+            } else if (ph.mode == MODE_GS) {
+                // item table: 16 global element offsets (one per slot), then 8 smem block bases
+                const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
+                for (int it = warp; it < ph.n_items; it += kWarps) {
+                    const int32_t *tab = ph.items + it * 24;
+                    uint4 raw[4][2];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int off = __ldg(tab + q * ph.lane_step + ph.j_off[j]);
+                        raw[j][0] = ldg128_stream(xA + off);
+                        raw[j][1] = ldg128_stream(xB + off);
+                    }
+                    uint32_t mats[8][4];
+                    octet_mma16<true>(raw, ph.bfrag + (size_t)it * 256 + lane, mats);
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const uint32_t addr = sbase + 2u * (uint32_t)(mrow * pitch + __ldg(tab + 16 + e) + mcol);
+                        stmatrix_x4(addr, mats[e][0], mats[e][1], mats[e][2], mats[e][3]);
+                    }
+                }
+            } else {   // MODE_CG
+                const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
+                for (int it = warp; it < ph.n_items; it += kWarps) {
+                    const int32_t *tab = ph.items + it * 24;
+                    uint4 out[4][2];
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) {
+                        float acc[2][2][4];
+#pragma unroll
+                        for (int ee = 0; ee < 2; ++ee) {
+                            const int e = 2 * w + ee;
+                            const uint4 bf = __ldg(ph.bfrag + (size_t)it * 256 + e * 32 + lane);
+                            uint32_t a[4];
+                            ldmatrix_x4(a, sbase + 2u * (uint32_t)(mrow * pitch + __ldg(tab + 16 + e) + mcol));
+                            mma_k16(acc[ee][0], a, bf.x, bf.y);
+                            mma_k16(acc[ee][1], a, bf.z, bf.w);
+                        }
+#pragma unroll
+                        for (int k = 0; k < 2; ++k)
+#pragma unroll
+                            for (int i = 0; i < 2; ++i)
+#pragma unroll
+                                for (int h = 0; h < 2; ++h)
+                                    set_word(out[i + 2 * k][h], w, pack_bf16(acc[0][k][i + 2 * h], acc[1][k][i + 2 * h]));
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const int off = __ldg(tab + q * ph.lane_step + ph.j_off[j]);
+                        if (okA) stg128(xA + off, out[j][0]);
+                        if (okB) stg128(xB + off, out[j][1]);
+                    }
+                }
+            }
+            __syncthreads();
+        }
+
+        if (P.copy_out) {
+            const int chunks = d >> 3;
+            for (int idx = threadIdx.x; idx < kTileRows * chunks; idx += kThreads) {
+                const int r = idx / chunks, c = idx - r * chunks;
+                if (row0 + r < n_rows) {
+                    const uint4 v = lds128(sbase + 2u * (uint32_t)(r * pitch + __ldg(P.chunk_phys + c)));
+                    stg128(x + (row0 + r) * d + 8 * c, v);
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+}  // namespace
+
+// ----------------------------------------------------------------------------- host
+
+struct FastPlan {
+    FastParams fwd{}, bwd{};
+    size_t smem_bytes = 0;
+    std::vector<void *> dev_allocs;
+    int max_ctas = 0;
+};
+
+namespace {
+
+struct HostPhase {
+    int t0, t1;          // stages [t0, t1)
+    int B;               // fused block size
+    int64_t S;           // natural stride of the phase (= s_{t0})
+    int64_t W;           // shared-memory element stride of the phase's local index
+    int lane_mult;       // 1 or 2
+};
+
+uint16_t f2bf(double v) {
+    const float f = (float)v;
+    uint32_t u;
+    std::memcpy(&u, &f, 4);
+    const uint32_t r = u + 0x7FFFu + ((u >> 16) & 1u);
+    return (uint16_t)(r >> 16);
+}
+
+// Fused block of phase hp for the block whose coordinates are base + r*S (r < B):
+// F[r_in][r_out] in fp64, the product of the phase's stages restricted to those coordinates.
+void fused_block(const harp_plan *plan, const HostPhase &hp, int64_t base, std::vector<double> &F) {
+    const int B = hp.B;
+    F.assign((size_t)B * B, 0.0);
+    for (int r = 0; r < B; ++r) F[(size_t)r * B + r] = 1.0;
+    std::vector<double> tmp((size_t)B * B);
+    for (int t = hp.t0; t < hp.t1; ++t) {
+        const int b = plan->st.b[t];
+        const int64_t s = plan->st.s[t];
+        const int64_t ls = s / hp.S;                     // local stride of this stage's digit
+        const float *Kt = plan->h_blocks.data() + plan->st.off[t];
+        std::fill(tmp.begin(), tmp.end(), 0.0);
+        for (int r = 0; r < B; ++r) {                    // r = output local index
+            const int digit = (int)((r / ls) % b);
+            const int r_base = r - digit * (int)ls;
+            const int64_t pos = base + (int64_t)r_base * hp.S;      // coordinate with the digit zeroed
+            const int64_t alpha = pos / ((int64_t)b * s), beta = pos % s;
+            const float *Kc = Kt + (alpha * s + beta) * b * b;
+            for (int i = 0; i < b; ++i) {                // input digit
+                const int r_in = r_base + i * (int)ls;
+                const double k = (double)Kc[i * b + digit];
+                for (int row = 0; row < B; ++row) tmp[(size_t)row * B + r] += F[(size_t)row * B + r_in] * k;
+            }
+        }
+        F.swap(tmp);
+    }
+}
+
+// slot maps: k-slot (or n-slot) index 0..B-1 of the MMA operand -> block-local index r
+int contig_slot(int kappa) { return kappa; }
+int strided_slot(int kappa, int B, int lane_mult) {
+    const int qq = (kappa & 7) >> 1, i = kappa & 1, k = kappa >> 3;
+    const int j = i + 2 * k;
+    if (B == 16) {
+        static const int joff1[4] = {0, 4, 8, 12}, joff2[4] = {0, 1, 8, 9};
+        return lane_mult * qq + (lane_mult == 1 ? joff1[j] : joff2[j]);
+    }
+    static const int joff1[2] = {0, 4}, joff2[2] = {0, 1};
+    return lane_mult * qq + (lane_mult == 1 ? joff1[j] : joff2[j]);
+}
+
+template <typename T>
+T *upload(FastPlan *fp, const std::vector<T> &v, harp_status_t &st) {
+    if (st != HARP_OK) return nullptr;
+    void *p = nullptr;
+    if (cudaMalloc(&p, std::max<size_t>(16, v.size() * sizeof(T))) != cudaSuccess) { st = HARP_ERR_ALLOC; return nullptr; }
+    fp->dev_allocs.push_back(p);
+    if (!v.empty() && cudaMemcpy(p, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) st = HARP_ERR_CUDA;
+    return static_cast<T *>(p);
+}
+
+}  // namespace
+
+harp_status_t harp_fast_build(harp_plan *plan) {
+    const int64_t d = plan->d;
+    const int m = plan->st.m;
+    if (d % 8 != 0) return HARP_ERR_UNSUPPORTED;
+
+    // ---- group stages into phases with fused size 8 or 16
+    std::vector<HostPhase> phases;
+    {
+        int t = 0;
+        while (t < m) {
+            int64_t prod = 1;
+            int t1 = t;
+            while (t1 < m && prod * plan->st.b[t1] <= 16) prod *= plan->st.b[t1++];
+            if (prod != 8 && prod != 16) return HARP_ERR_UNSUPPORTED;
+            phases.push_back({t, t1, (int)prod, plan->st.s[t], 0, 1});
+            t = t1;
+        }
+    }
+    const int np = (int)phases.size();
+    if (np > kMaxPhases) return HARP_ERR_UNSUPPORTED;
+
+    // ---- shared-memory layout: local index r_p of phase p has element stride W_p
+    int64_t W = 1;
+    for (int p = 0; p < np; ++p) {
+        if (p > 0) {
+            W = (W + 7) / 8 * 8;
+            while (((W / 8) % 8) == 0 || ((W / 8) % 8) == 4) W += 8;
+            phases[p].lane_mult = ((W / 8) % 2 == 0) ? 1 : 2;
+        }
+        phases[p].W = W;
+        W *= phases[p].B;
+    }
+    int64_t pitch = (W + 7) / 8 * 8;
+    if ((pitch / 8) % 2 == 0) pitch += 8;
+    const size_t smem_bytes = (size_t)kTileRows * pitch * 2;
+    if (smem_bytes > 227u * 1024u) return HARP_ERR_UNSUPPORTED;
+
+    auto phys = [&](int64_t pos) {
+        int64_t o = 0;
+        for (int p = 0; p < np; ++p) o += ((pos / phases[p].S) % phases[p].B) * phases[p].W;
+        return o;
+    };
+
+    // ---- permutation structure
+    const bool identity = plan->h_perm.empty();
+    const int B0 = phases[0].B;
+    const int64_t nblk0 = d / B0;
+    std::vector<std::vector<int64_t>> octets;           // per item: the 8 first-phase blocks
+    if (!identity) {
+        if (B0 != 16) return HARP_ERR_UNSUPPORTED;
+        std::vector<int64_t> order((size_t)nblk0);
+        for (int64_t c = 0; c < nblk0; ++c) order[(size_t)c] = c;
+        const int32_t *pm = plan->h_perm.data();
+        std::sort(order.begin(), order.end(), [&](int64_t a, int64_t b) { return pm[a * B0] < pm[b * B0]; });
+        if (nblk0 % 8 != 0) return HARP_ERR_UNSUPPORTED;
+        for (int64_t i = 0; i < nblk0; i += 8) {
+            std::vector<int64_t> oc(order.begin() + i, order.begin() + i + 8);
+            for (int r = 0; r < B0; ++r) {
+                const int32_t s0 = pm[oc[0] * B0 + r];
+                if (s0 % 8 != 0) return HARP_ERR_UNSUPPORTED;
+                for (int e = 1; e < 8; ++e)
+                    if (pm[oc[(size_t)e] * B0 + r] != s0 + e) return HARP_ERR_UNSUPPORTED;
+            }
+            octets.push_back(oc);
+        }
+    }
+
+    FastPlan *fp = new (std::nothrow) FastPlan();
+    if (!fp) return HARP_ERR_ALLOC;
+    fp->smem_bytes = smem_bytes;
+    harp_status_t st = HARP_OK;
+
+    std::vector<int32_t> chunk_phys((size_t)(d / 8));
+    for (int64_t c = 0; c < d / 8; ++c) chunk_phys[(size_t)c] = (int32_t)phys(8 * c);
+    const int32_t *d_chunk = upload(fp, chunk_phys, st);
+
+    auto sign_v = [&](int64_t i) -> double {             // sign seen by coordinate i after the gather
+        if (plan->h_signs.empty()) return 1.0;
+        const int64_t src = identity ? i : plan->h_perm[(size_t)i];
+        return (double)plan->h_signs[(size_t)src];
+    };
+
+    for (int dir = 0; dir < 2; ++dir) {                  // 0 = forward, 1 = transpose
+        FastParams &P = dir == 0 ? fp->fwd : fp->bwd;
+        P.n_phases = np;
+        P.d = (int32_t)d;
+        P.pitch = (int32_t)pitch;
+        P.chunk_phys = d_chunk;
+        P.copy_in = (dir == 1 || identity) ? 1 : 0;
+        P.copy_out = (dir == 0 || identity) ? 1 : 0;
+        for (int k = 0; k < np && st == HARP_OK; ++k) {
+            const int p = dir == 0 ? k : np - 1 - k;     // phase executed k-th
+            const HostPhase &hp = phases[p];
+            PhaseDesc &D = P.ph[k];
+            const int B = hp.B;
+            int mode;
+            if (p == 0) mode = identity ? MODE_CC : (dir == 0 ? MODE_GS : MODE_CG);
+            else mode = MODE_SS;
+            D.mode = mode;
+            D.B = B;
+            // slot geometry of the strided side
+            const int lm = (p == 0) ? 1 : hp.lane_mult;
+            static const int joff1_16[4] = {0, 4, 8, 12}, joff2_16[4] = {0, 1, 8, 9};
+            static const int joff1_8[4] = {0, 4, 0, 0}, joff2_8[4] = {0, 1, 0, 0};
+            const int *jo = B == 16 ? (lm == 1 ? joff1_16 : joff2_16) : (lm == 1 ? joff1_8 : joff2_8);
+            if (mode == MODE_SS) {
+                D.lane_step = (int32_t)(lm * hp.W);
+                for (int j = 0; j < 4; ++j) D.j_off[j] = (int32_t)(jo[j] * hp.W);
+            } else {                                     // GS / CG index the item table by slot
+                D.lane_step = lm;
+                for (int j = 0; j < 4; ++j) D.j_off[j] = jo[j];
+            }
+            // enumerate items and the natural base coordinate of every block
+            std::vector<int32_t> items;
+            std::vector<int64_t> block_base;             // natural coordinate of r = 0, per block in item order
+            if (mode == MODE_CC) {
+                for (int64_t c = 0; c < nblk0; ++c) {
+                    items.push_back((int32_t)phys(c * B0));
+                    block_base.push_back(c * B0);
+                }
+            } else if (mode == MODE_SS) {
+                // all coordinates with r_p = 0 and r_0 a multiple of 8
+                const int64_t span = hp.S * B;
+                for (int64_t hi = 0; hi < d; hi += span)
+                    for (int64_t lo = 0; lo < hp.S; lo += 8) {
+                        items.push_back((int32_t)phys(hi + lo));
+                        for (int e = 0; e < 8; ++e) block_base.push_back(hi + lo + e);
+                    }
+            } else {
+                for (const auto &oc : octets) {
+                    for (int r = 0; r < 16; ++r) items.push_back(plan->h_perm[(size_t)(oc[0] * B0 + r)]);
+                    for (int e = 0; e < 8; ++e) {
+                        items.push_back((int32_t)phys(oc[(size_t)e] * B0));
+                        block_base.push_back(oc[(size_t)e] * B0);
+                    }
+                }
+            }
+            D.n_items = (int32_t)(mode == MODE_CC ? nblk0 : (mode == MODE_SS ? (int64_t)items.size() : (int64_t)octets.size()));
+            // every address the kernel will form from these tables must stay inside the tile / the row
+            {
+                bool ok = true;
+                if (mode == MODE_CC) {
+                    for (int32_t b : items) ok = ok && b >= 0 && b % 8 == 0 && b + B <= pitch;
+                } else if (mode == MODE_SS) {
+                    const int nj = B == 16 ? 4 : 2;
+                    for (int32_t b : items)
+                        for (int qq = 0; qq < 4; ++qq)
+                            for (int j = 0; j < nj; ++j) {
+                                const int64_t o = (int64_t)b + (int64_t)qq * D.lane_step + D.j_off[j];
+                                ok = ok && b >= 0 && o % 8 == 0 && o + 8 <= pitch;
+                            }
+                } else {
+                    for (size_t i = 0; i < items.size(); i += 24) {
+                        for (int r = 0; r < 16; ++r) ok = ok && items[i + r] >= 0 && items[i + r] % 8 == 0 && items[i + r] + 8 <= d;
+                        for (int e = 0; e < 8; ++e) ok = ok && items[i + 16 + e] >= 0 && items[i + 16 + e] % 8 == 0 && items[i + 16 + e] + 16 <= pitch;
+                    }
+                }
+                if (!ok) { st = HARP_ERR_UNSUPPORTED; break; }
+            }
+            D.items = upload(fp, items, st);
+            // fragments
+            const bool in_strided = (mode == MODE_SS || mode == MODE_GS);
+            const bool out_strided = (mode == MODE_SS || mode == MODE_CG);
+            const int words_per_lane = B == 16 ? 4 : 1;
+            std::vector<uint32_t> frag(block_base.size() * 32 * words_per_lane);
+            std::vector<double> F;
+            for (size_t bi = 0; bi < block_base.size(); ++bi) {
+                fused_block(plan, hp, block_base[bi], F);
+                // G[r_in][r_out]: the matrix this phase applies in this direction, signs folded in
+                auto G = [&](int rin, int rout) -> double {
+                    double v = dir == 0 ? F[(size_t)rin * B + rout] : F[(size_t)rout * B + rin];
+                    if (p == 0 && dir == 0) v *= sign_v(block_base[bi] + rin);
+                    if (p == 0 && dir == 1) v *= sign_v(block_base[bi] + rout);
+                    return v;
+                };
+                auto kin = [&](int kappa) { return in_strided ? strided_slot(kappa, B, lm) : contig_slot(kappa); };
+                auto nout = [&](int nu) { return out_strided ? strided_slot(nu, B, lm) : contig_slot(nu); };
+                for (int lane = 0; lane < 32; ++lane) {
+                    const int gg = lane >> 2, qq = lane & 3;
+                    uint32_t *dst = frag.data() + (bi * 32 + lane) * words_per_lane;
+                    if (B == 16) {
+                        for (int nt = 0; nt < 2; ++nt) {
+                            const int n = nout(8 * nt + gg);
+                            const uint32_t b0 = f2bf(G(kin(2 * qq), n)) | ((uint32_t)f2bf(G(kin(2 * qq + 1), n)) << 16);
+                            const uint32_t b1 = f2bf(G(kin(2 * qq + 8), n)) | ((uint32_t)f2bf(G(kin(2 * qq + 9), n)) << 16);
+                            dst[2 * nt] = b0;
+                            dst[2 * nt + 1] = b1;
+                        }
+                    } else {
+                        const int n = nout(gg);
+                        dst[0] = f2bf(G(kin(2 * qq), n)) | ((uint32_t)f2bf(G(kin(2 * qq + 1), n)) << 16);
+                    }
+                }
+            }
+            D.bfrag = reinterpret_cast<const uint4 *>(upload(fp, frag, st));
+        }
+    }
+    if (st == HARP_OK) {
+        if (cudaFuncSetAttribute(harp_fast_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+            st = HARP_ERR_CUDA;
+        int dev = 0, sms = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        fp->max_ctas = sms > 0 ? sms : 148;
+    }
+    plan->fast = fp;
+    if (st != HARP_OK) {
+        cudaGetLastError();
+        harp_fast_destroy(plan);
+        return st;
+    }
+    return HARP_OK;
+}
+
+void harp_fast_destroy(harp_plan *plan) {
+    if (!plan->fast) return;
+    for (void *p : plan->fast->dev_allocs) cudaFree(p);
+    delete plan->fast;
+    plan->fast = nullptr;
+}
+
+harp_status_t harp_fast_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype, int transpose,
+                              cudaStream_t stream) {
+    const FastPlan *fp = plan->fast;
+    if (!fp || dtype != HARP_BF16) return HARP_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(x) & 15u) != 0) return HARP_ERR_UNSUPPORTED;
+    const int64_t n_tiles = (n_rows + kTileRows - 1) / kTileRows;
+    const int grid = (int)std::min<int64_t>(n_tiles, fp->max_ctas);
+    harp_fast_kernel<<<grid, kThreads, fp->smem_bytes, stream>>>(static_cast<__nv_bfloat16 *>(x), n_rows, n_tiles,
+                                                                 transpose ? fp->bwd : fp->fwd);
+    g_harp_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? HARP_OK : HARP_ERR_CUDA;
 }

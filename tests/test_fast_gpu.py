@@ -1,0 +1,50 @@
+"""Tensor-core path (explicit HARP_KERNEL_FAST) against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2605_29843_b200 as harp
+from oracle import harp_oracle as orc
+from paper_2605_29843_b200 import workloads as wl
+from harp_testlib import TOL, gpu_apply, host_rows, promote
+
+pytestmark = pytest.mark.gpu
+
+SUPPORTED = [
+    ((4, 4), "identity"), ((4, 4, 4, 4), "identity"), ((4,) * 6, "identity"), ((4,) * 6, "digit_reversal"),
+    ((2,) * 11, "identity"), ((2,) * 11, "digit_reversal"), ((8, 8), "identity"), ((8, 8, 8, 8), "identity"),
+    ((16, 16, 8), "identity"), ((16, 16, 8), "digit_reversal"), ((2, 8, 4, 4, 8), "identity"),
+    ((4, 4, 2, 2, 2, 2, 16), "digit_reversal"), ((16, 16, 16), "digit_reversal"),
+]
+
+
+@pytest.mark.parametrize("radices,perm", SUPPORTED)
+@pytest.mark.parametrize("kind", ["qr", "identity"])
+def test_fast_kernel_matches_oracle(radices, perm, kind):
+    spec = wl.make_plan(23, int(np.prod(radices)), radices, kind, perm=perm, signs=True)
+    oplan = orc.OraclePlan.from_spec(spec)
+    plan = harp.plan_from_spec(spec)
+    rng = np.random.default_rng(8)
+    for n_rows in (1, 16, 37, 600):
+        xh = host_rows(rng.standard_normal((n_rows, spec.d)), "bf16")
+        x64 = promote(xh, "bf16")
+        for tr in (False, True):
+            got, guards = gpu_apply(plan, xh, "bf16", tr, harp.KERNEL_FAST)
+            want = orc.transpose(oplan, x64) if tr else orc.forward(oplan, x64)
+            assert guards
+            if kind == "identity":
+                assert np.array_equal(got, want)            # sign + gather must be bit exact
+            else:
+                assert orc.rel_err_rows(got, want) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("radices,perm,dtype", [((16, 16, 8, 7), "identity", "bf16"), ((4,) * 6, "random", "bf16"),
+                                                ((4,) * 6, "identity", "f32"), ((2,) * 9, "identity", "bf16")])
+def test_fast_kernel_reports_unsupported(radices, perm, dtype):
+    spec = wl.make_plan(3, int(np.prod(radices)), radices, "qr", perm=perm)
+    plan = harp.plan_from_spec(spec)
+    x = torch.zeros((16, spec.d), device="cuda", dtype=torch.float32 if dtype == "f32" else torch.bfloat16)
+    st = harp.lib().harp_apply_ex(plan.handle, x.data_ptr(), 16, 0 if dtype == "f32" else 1, 0, harp.KERNEL_FAST, None)
+    assert st == harp.HARP_ERR_UNSUPPORTED
+    harp.apply_(plan, x)                                    # AUTO still works (generic kernel)
+    torch.cuda.synchronize()
