@@ -52,7 +52,12 @@ typedef enum {
 typedef enum { HARP_F32 = 0, HARP_BF16 = 1 } harp_dtype_t;
 
 /* Kernel families; HARP_KERNEL_AUTO lets the library choose. */
-typedef enum { HARP_KERNEL_AUTO = 0, HARP_KERNEL_GENERIC = 1, HARP_KERNEL_FAST = 2 } harp_kernel_t;
+typedef enum {
+    HARP_KERNEL_AUTO = 0,
+    HARP_KERNEL_GENERIC = 1,   /* CUDA cores, any plan                                   */
+    HARP_KERNEL_FAST = 2,      /* tensor cores, whole rows per CTA                       */
+    HARP_KERNEL_SPLIT = 3      /* tensor cores, two passes over column groups (wide rows) */
+} harp_kernel_t;
 
 /* Build a processor (Eq. 6-9 of the paper; Algorithm 1 lines 2 and 7-8 for the stride
  * and block-kernel layout).

@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libharp.so")
 
 HARP_F32, HARP_BF16 = 0, 1
-KERNEL_AUTO, KERNEL_GENERIC, KERNEL_FAST = 0, 1, 2
+KERNEL_AUTO, KERNEL_GENERIC, KERNEL_FAST, KERNEL_SPLIT = 0, 1, 2, 3
 HARP_OK = 0
 HARP_ERR_UNSUPPORTED = 8
 

@@ -124,6 +124,10 @@ extern "C" harp_status_t harp_plan_create(harp_plan_t **out, int64_t d, int32_t 
         harp_status_t fs = harp_fast_build(p);
         if (fs != HARP_OK && fs != HARP_ERR_UNSUPPORTED) st = fs;
     }
+    if (st == HARP_OK) {
+        harp_status_t fs = harp_split_build(p);
+        if (fs != HARP_OK && fs != HARP_ERR_UNSUPPORTED) st = fs;
+    }
     if (st != HARP_OK) {
         cudaGetLastError();
         harp_plan_destroy(p);
@@ -138,6 +142,7 @@ extern "C" void harp_plan_destroy(harp_plan_t *p) {
     {
         DeviceGuard g(p->device);
         harp_fast_destroy(p);
+        harp_split_destroy(p);
         for (int i = 0; i < 2; ++i) {
             if (p->stage_stream[i]) { cudaStreamSynchronize(p->stage_stream[i]); cudaStreamDestroy(p->stage_stream[i]); }
             if (p->stage_buf[i]) cudaFree(p->stage_buf[i]);
@@ -156,7 +161,8 @@ extern "C" harp_status_t harp_apply_ex(const harp_plan_t *plan, void *x, int64_t
     if (!plan) return HARP_ERR_NULL;
     if (dtype != HARP_F32 && dtype != HARP_BF16) return HARP_ERR_BAD_DTYPE;
     if (n_rows < 0) return HARP_ERR_BAD_DIM;
-    if (kernel != HARP_KERNEL_AUTO && kernel != HARP_KERNEL_GENERIC && kernel != HARP_KERNEL_FAST)
+    if (kernel != HARP_KERNEL_AUTO && kernel != HARP_KERNEL_GENERIC && kernel != HARP_KERNEL_FAST &&
+        kernel != HARP_KERNEL_SPLIT)
         return HARP_ERR_UNSUPPORTED;
     if (n_rows == 0) return HARP_OK;
     if (!x) return HARP_ERR_NULL;
@@ -165,7 +171,10 @@ extern "C" harp_status_t harp_apply_ex(const harp_plan_t *plan, void *x, int64_t
     transpose = transpose ? 1 : 0;
     if (kernel == HARP_KERNEL_GENERIC) return harp_generic_apply(plan, x, n_rows, dtype, transpose, s);
     if (kernel == HARP_KERNEL_FAST) return harp_fast_apply(plan, x, n_rows, dtype, transpose, s);
+    if (kernel == HARP_KERNEL_SPLIT) return harp_split_apply(plan, x, n_rows, dtype, transpose, s);
     harp_status_t st = harp_fast_apply(plan, x, n_rows, dtype, transpose, s);
+    if (st != HARP_ERR_UNSUPPORTED) return st;
+    st = harp_split_apply(plan, x, n_rows, dtype, transpose, s);
     if (st != HARP_ERR_UNSUPPORTED) return st;
     return harp_generic_apply(plan, x, n_rows, dtype, transpose, s);
 }

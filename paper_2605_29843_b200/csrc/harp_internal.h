@@ -20,7 +20,8 @@ struct StageTable {
     int64_t off[HARP_MAX_STAGES];     // offset (in floats) of stage t in the block array
 };
 
-struct FastPlan;   // tensor-core path data (harp_fast.cu)
+struct FastPlan;   // tensor-core path data, whole rows per CTA (harp_fast.cu)
+struct SplitPlan;  // tensor-core path data, two passes over column groups (harp_split.cu)
 
 struct harp_plan {
     int64_t d = 0;
@@ -35,6 +36,7 @@ struct harp_plan {
     std::vector<int8_t> h_signs;
     std::vector<float> h_blocks;
     FastPlan *fast = nullptr;
+    SplitPlan *split = nullptr;
     // staging owned by harp_apply_host
     void *stage_buf[2] = {nullptr, nullptr};
     int64_t stage_bytes = 0;
@@ -53,6 +55,12 @@ harp_status_t harp_fast_build(harp_plan *plan);     // HARP_OK or HARP_ERR_UNSUP
 void harp_fast_destroy(harp_plan *plan);
 harp_status_t harp_fast_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype,
                               int transpose, cudaStream_t stream);
+
+// tensor-core path for wide rows (harp_split.cu)
+harp_status_t harp_split_build(harp_plan *plan);
+void harp_split_destroy(harp_plan *plan);
+harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype,
+                               int transpose, cudaStream_t stream);
 
 // out-of-place matrix transpose, rows x cols -> cols x rows (harp_two_sided.cu)
 harp_status_t harp_transpose_matrix(const void *src, void *dst, int64_t rows, int64_t cols,

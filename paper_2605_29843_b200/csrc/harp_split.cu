@@ -1,0 +1,532 @@
+// Tensor-core path for wide rows (bf16, identity permutation): two passes over column groups.
+//
+// A row of d = S_mid * U coordinates is seen as a U x S_mid array.  The stages with stride
+// below S_mid ("lower") only mix coordinates inside one slab of S_mid contiguous
+// coordinates; the remaining ("upper") stages only mix coordinates that share the position
+// l inside their slab.  So the transform is done in two passes, each of which gives a CTA
+// a column group and many rows:
+//   pass 1: column group = one slab (S_mid contiguous coordinates), lower stages;
+//   pass 2: column group = Lw neighbouring positions l in every slab (U segments of Lw
+//           coordinates), upper stages.
+// Within a pass a CTA keeps the fused block kernels of its column group resident in shared
+// memory for all the rows it processes (they are never re-read from L2), and works on
+// tiles of 16*MT rows: coalesced cp.async in, phases as batches of small mma.sync products
+// with the rows as the M dimension (see harp_fast.cu for the operand handling), coalesced
+// stores out.  Tiles are small, so several CTAs share an SM and their copies overlap with
+// each other's arithmetic.
+//
+// The host walks over the batch in row chunks small enough to stay in L2 and launches
+// pass 1 and pass 2 for a chunk back to back, so that the second pass finds the rows in L2:
+// HBM sees one read and one write per row; only L2 sees two.
+//
+// Radices that do not fill an 8- or 16-wide block (7, 2, ...) are zero-padded inside the
+// fragments; padded slots read a valid coordinate and are never stored.
+#include <algorithm>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "harp_internal.h"
+#include "harp_mma.cuh"
+#include "harp_fuse.h"
+
+using namespace harp_fuse;
+
+namespace {
+
+constexpr int kSplitThreads = 256;
+constexpr int kSplitWarps = kSplitThreads / 32;
+constexpr int kMaxSplitPhases = 6;
+
+struct SplitPhase {
+    int32_t mode;              // 0 = contiguous blocks (ldmatrix), 1 = strided blocks, eight per item
+    int32_t B, B_real;         // operand width (8 or 16) and number of real coordinates in a block
+    int32_t lane_step;         // element offset between the slots of lanes q and q+1
+    int32_t j_off[4];          // element offsets of a lane's slots
+    int32_t lm, jr[4];         // local index of slot j of lane q is lm*q + jr[j]
+    int32_t items_off, n_items;
+    int32_t bfrag_off;         // word offset of the phase's fragments inside a column group's block
+};
+
+struct SplitPass {
+    int32_t n_phases, n_cg, n_chunks, pitch, MT;
+    int32_t cg_stride;         // global element offset between column groups
+    int32_t row_stride;        // d
+    int32_t chunk_off;         // tables[chunk_off + 2c] = global offset, [.. + 1] = smem offset of 16-byte chunk c
+    const int32_t *tables;
+    int32_t tables_len;
+    const uint32_t *bfrag;     // [column group][bfrag_words]
+    int32_t bfrag_words;
+    SplitPhase ph[kMaxSplitPhases];
+};
+
+__device__ __forceinline__ uint32_t lds32(uint32_t addr) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+
+__global__ void __launch_bounds__(kSplitThreads, 2)
+harp_split_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_end, SplitPass P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const uint32_t sbase = smem_u32(smem_raw);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, q = lane & 3;
+    const int pitch = P.pitch, MT = P.MT;
+    const int tile_rows = 16 * MT;
+    const size_t tile_bytes = (size_t)tile_rows * pitch * 2;
+    int32_t *tab_s = reinterpret_cast<int32_t *>(smem_raw + tile_bytes);
+    const uint32_t bf_s = sbase + (uint32_t)((tile_bytes + (size_t)P.tables_len * 4 + 15) / 16 * 16);
+
+    const int cg = blockIdx.x % P.n_cg, part = blockIdx.x / P.n_cg, n_parts = gridDim.x / P.n_cg;
+    // resident data of this column group: tables and fragments
+    for (int i = threadIdx.x; i < P.tables_len; i += kSplitThreads) tab_s[i] = __ldg(P.tables + i);
+    {
+        const uint32_t *src = P.bfrag + (size_t)cg * P.bfrag_words;
+        for (int i = threadIdx.x * 4; i < P.bfrag_words; i += kSplitThreads * 4) cp_async16(bf_s + 4u * i, src + i);
+    }
+    cp_async_wait_all();
+    __syncthreads();
+
+    __nv_bfloat16 *xg = x + (size_t)cg * P.cg_stride;
+    const int64_t n_rows = row_end - row_begin;
+    const int64_t n_tiles = (n_rows + tile_rows - 1) / tile_rows;
+    const int32_t *cmap = tab_s + P.chunk_off;
+    const int64_t rs = P.row_stride;
+
+    for (int64_t tile = part; tile < n_tiles; tile += n_parts) {
+        const int64_t row0 = row_begin + tile * tile_rows;
+        const int64_t last = row_end - 1;
+        // rows past the end are computed on a copy of the last row and never stored
+        for (int idx = threadIdx.x; idx < tile_rows * P.n_chunks; idx += kSplitThreads) {
+            const int r = idx / P.n_chunks, ch = idx - r * P.n_chunks;
+            const int64_t row = min(row0 + r, last);
+            cp_async16(sbase + 2u * (uint32_t)(r * pitch + cmap[2 * ch + 1]), xg + row * rs + cmap[2 * ch]);
+        }
+        cp_async_wait_all();
+        __syncthreads();
+
+        for (int p = 0; p < P.n_phases; ++p) {
+            const SplitPhase &ph = P.ph[p];
+            const int n_work = ph.n_items * MT;
+            if (ph.mode == 0) {
+                if (ph.B == 16) {
+                    const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
+#pragma unroll 2
+                    for (int w = warp; w < n_work; w += kSplitWarps) {
+                        const int it = w / MT, mt = w - it * MT;
+                        const uint32_t addr = sbase + 2u * (uint32_t)((mt * 16 + mrow) * pitch + tab_s[ph.items_off + it] + mcol);
+                        const uint4 bf = lds128(bf_s + 4u * (uint32_t)(ph.bfrag_off + (it * 32 + lane) * 4));
+                        uint32_t a[4];
+                        ldmatrix_x4(a, addr);
+                        float c0[4], c1[4];
+                        mma_k16(c0, a, bf.x, bf.y);
+                        mma_k16(c1, a, bf.z, bf.w);
+                        stmatrix_x4(addr, pack_bf16(c0[0], c0[1]), pack_bf16(c0[2], c0[3]), pack_bf16(c1[0], c1[1]),
+                                    pack_bf16(c1[2], c1[3]));
+                    }
+                } else {
+                    const int mrow2 = lane & 15;
+#pragma unroll 2
+                    for (int w = warp; w < n_work; w += kSplitWarps) {
+                        const int it = w / MT, mt = w - it * MT;
+                        const uint32_t addr = sbase + 2u * (uint32_t)((mt * 16 + mrow2) * pitch + tab_s[ph.items_off + it]);
+                        const uint32_t bf = lds32(bf_s + 4u * (uint32_t)(ph.bfrag_off + it * 32 + lane));
+                        uint32_t a[2];
+                        ldmatrix_x2(a, addr);
+                        float c0[4];
+                        mma_k8(c0, a, bf);
+                        stmatrix_x2(addr, pack_bf16(c0[0], c0[1]), pack_bf16(c0[2], c0[3]));
+                    }
+                }
+            } else if (ph.B == 16) {
+                // per-lane slot offsets; padded slots read slot 0 and are not stored
+                uint32_t so[4];
+                bool ok[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    ok[j] = ph.lm * q + ph.jr[j] < ph.B_real;
+                    so[j] = ok[j] ? 2u * (uint32_t)(q * ph.lane_step + ph.j_off[j]) : 0u;
+                }
+                for (int w = warp; w < n_work; w += kSplitWarps) {
+                    const int it = w / MT, mt = w - it * MT;
+                    const uint32_t a0 = sbase + 2u * (uint32_t)((mt * 16 + g) * pitch + tab_s[ph.items_off + it]);
+                    const uint32_t a1 = a0 + 2u * (uint32_t)(8 * pitch);
+                    uint4 raw[4][2], bf[8];
+                    uint32_t unused[8][4];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) bf[e] = lds128(bf_s + 4u * (uint32_t)(ph.bfrag_off + ((it * 8 + e) * 32 + lane) * 4));
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        raw[j][0] = lds128(a0 + so[j]);
+                        raw[j][1] = lds128(a1 + so[j]);
+                    }
+                    octet_mma16<true>(raw, bf, unused);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (ok[j]) {
+                            sts128(a0 + so[j], raw[j][0]);
+                            sts128(a1 + so[j], raw[j][1]);
+                        }
+                    }
+                }
+            } else {
+                uint32_t so[2];
+                bool ok[2];
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    ok[j] = ph.lm * q + ph.jr[j] < ph.B_real;
+                    so[j] = ok[j] ? 2u * (uint32_t)(q * ph.lane_step + ph.j_off[j]) : 0u;
+                }
+                for (int w = warp; w < n_work; w += kSplitWarps) {
+                    const int it = w / MT, mt = w - it * MT;
+                    const uint32_t a0 = sbase + 2u * (uint32_t)((mt * 16 + g) * pitch + tab_s[ph.items_off + it]);
+                    const uint32_t a1 = a0 + 2u * (uint32_t)(8 * pitch);
+                    uint4 raw[2][2];
+                    uint32_t bf[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) bf[e] = lds32(bf_s + 4u * (uint32_t)(ph.bfrag_off + (it * 8 + e) * 32 + lane));
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        raw[j][0] = lds128(a0 + so[j]);
+                        raw[j][1] = lds128(a1 + so[j]);
+                    }
+                    octet_mma8(raw, bf);
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        if (ok[j]) {
+                            sts128(a0 + so[j], raw[j][0]);
+                            sts128(a1 + so[j], raw[j][1]);
+                        }
+                    }
+                }
+            }
+            __syncthreads();
+        }
+
+        for (int idx = threadIdx.x; idx < tile_rows * P.n_chunks; idx += kSplitThreads) {
+            const int r = idx / P.n_chunks, ch = idx - r * P.n_chunks;
+            if (row0 + r < row_end) {
+                const uint4 v = lds128(sbase + 2u * (uint32_t)(r * pitch + cmap[2 * ch + 1]));
+                stg128(xg + (row0 + r) * rs + cmap[2 * ch], v);
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------------------------- host
+
+struct PassHost {
+    SplitPass fwd{}, bwd{};
+    size_t smem_bytes = 0;
+    bool present = false;
+};
+
+}  // namespace
+
+struct SplitPlan {
+    PassHost pass[2];          // [0] lower stages on slabs, [1] upper stages on position groups
+    std::vector<void *> dev_allocs;
+    int64_t chunk_rows = 0;    // rows per L2-resident chunk
+    int sms = 148;
+};
+
+namespace {
+
+struct GPhase {                // a fused group of stages
+    int t0, t1;
+    int B, B_real;
+    int64_t S;                 // natural stride
+};
+
+template <typename T>
+T *upload_s(SplitPlan *sp, const std::vector<T> &v, harp_status_t &st) {
+    if (st != HARP_OK) return nullptr;
+    void *p = nullptr;
+    if (cudaMalloc(&p, std::max<size_t>(16, v.size() * sizeof(T))) != cudaSuccess) { st = HARP_ERR_ALLOC; return nullptr; }
+    sp->dev_allocs.push_back(p);
+    if (!v.empty() && cudaMemcpy(p, v.data(), v.size() * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) st = HARP_ERR_CUDA;
+    return static_cast<T *>(p);
+}
+
+// One pass.  `phs`: the pass's phases.  Tile coordinates: an innermost index of `inner` positions
+// (stride 1 in memory, not mixed by this pass unless it is phase 0 of pass 1) followed by the
+// phases' local indices.  For pass 1, inner = 1 and phase 0 is contiguous; for pass 2, inner = Lw.
+harp_status_t build_pass(const harp_plan *plan, SplitPlan *sp, PassHost &ph_out, const std::vector<GPhase> &phs, bool lower,
+                         int64_t S_mid, int64_t U, int inner) {
+    const int64_t d = plan->d;
+    const int np = (int)phs.size();
+    if (np == 0 || np > kMaxSplitPhases) return HARP_ERR_UNSUPPORTED;
+    // ---- layout of a tile row
+    std::vector<int64_t> W((size_t)np);
+    std::vector<int> lm((size_t)np, 1);
+    int64_t ext = inner;
+    for (int p = 0; p < np; ++p) {
+        if (!(lower && p == 0)) {
+            ext = (ext + 7) / 8 * 8;
+            while (((ext / 8) % 8) == 0 || ((ext / 8) % 8) == 4) ext += 8;
+            lm[(size_t)p] = ((ext / 8) % 2 == 0) ? 1 : 2;
+        }
+        W[(size_t)p] = ext;
+        ext *= phs[(size_t)p].B_real;
+    }
+    int64_t pitch = (ext + 7) / 8 * 8;
+    if ((pitch / 8) % 2 == 0) pitch += 8;
+    // local strides of the phases inside the tile's own coordinate system
+    // pass 1: tile coordinate t in [0, S_mid): local index of phase p = (t / S_p) % B_real
+    // pass 2: tile coordinate (l', u): local index of phase p = (u / (S_p / S_mid)) % B_real
+    auto phys = [&](int64_t lpos, int64_t u) {       // lpos: position inside the inner run / slab
+        int64_t o = 0;
+        if (lower) {
+            for (int p = 0; p < np; ++p) o += ((lpos / phs[(size_t)p].S) % phs[(size_t)p].B_real) * W[(size_t)p];
+        } else {
+            o = lpos;
+            for (int p = 0; p < np; ++p) o += ((u / (phs[(size_t)p].S / S_mid)) % phs[(size_t)p].B_real) * W[(size_t)p];
+        }
+        return o;
+    };
+    const int n_cg = lower ? (int)U : (int)(S_mid / inner);
+    const int n_chunks = lower ? (int)(S_mid / 8) : (int)(U * inner / 8);
+    // rows per tile: as many 16-row groups as fit ~40 KB
+    int MT = (int)std::max<int64_t>(1, std::min<int64_t>(4, (40 * 1024) / (pitch * 2 * 16)));
+
+    // ---- tables: chunk map, then items per phase (identical for all column groups and both directions)
+    std::vector<int32_t> tables;
+    for (int c = 0; c < n_chunks; ++c) {
+        if (lower) {
+            tables.push_back(8 * c);
+            tables.push_back((int32_t)phys(8 * c, 0));
+        } else {
+            const int per = inner / 8;
+            const int64_t u = c / per, lc = (c % per) * 8;
+            tables.push_back((int32_t)(u * S_mid + lc));
+            tables.push_back((int32_t)phys(lc, u));
+        }
+    }
+    struct ItemSet { std::vector<int32_t> bases; std::vector<int64_t> block_rel; int mode; };   // block_rel: (lpos, u) packed
+    std::vector<ItemSet> sets((size_t)np);
+    for (int p = 0; p < np; ++p) {
+        const GPhase &gp = phs[(size_t)p];
+        ItemSet &is = sets[(size_t)p];
+        if (lower && p == 0) {
+            is.mode = 0;
+            if (gp.B != gp.B_real) return HARP_ERR_UNSUPPORTED;
+            for (int64_t c = 0; c < S_mid / gp.B; ++c) {
+                is.bases.push_back((int32_t)phys(c * gp.B, 0));
+                is.block_rel.push_back(c * gp.B);
+            }
+        } else if (lower) {
+            is.mode = 1;
+            const int64_t span = gp.S * gp.B_real;
+            for (int64_t hi = 0; hi < S_mid; hi += span)
+                for (int64_t lo = 0; lo < gp.S; lo += 8) {
+                    is.bases.push_back((int32_t)phys(hi + lo, 0));
+                    for (int e = 0; e < 8; ++e) is.block_rel.push_back(hi + lo + e);
+                }
+        } else {
+            is.mode = 1;
+            const int64_t su = gp.S / S_mid, span = su * gp.B_real;      // in units of u
+            for (int64_t hi = 0; hi < U; hi += span)
+                for (int64_t lo = 0; lo < su; ++lo)
+                    for (int64_t lc = 0; lc < inner; lc += 8) {
+                        is.bases.push_back((int32_t)phys(lc, hi + lo));
+                        for (int e = 0; e < 8; ++e) is.block_rel.push_back((hi + lo) * S_mid + lc + e);   // relative natural coordinate
+                    }
+        }
+    }
+
+    static const int joff1_16[4] = {0, 4, 8, 12}, joff2_16[4] = {0, 1, 8, 9};
+    static const int joff1_8[4] = {0, 4, 0, 0}, joff2_8[4] = {0, 1, 0, 0};
+    harp_status_t st = HARP_OK;
+    for (int dir = 0; dir < 2 && st == HARP_OK; ++dir) {
+        SplitPass &P = dir == 0 ? ph_out.fwd : ph_out.bwd;
+        P.n_phases = np;
+        P.n_cg = n_cg;
+        P.n_chunks = n_chunks;
+        P.pitch = (int32_t)pitch;
+        P.MT = MT;
+        P.cg_stride = lower ? (int32_t)S_mid : inner;
+        P.row_stride = (int32_t)d;
+        P.chunk_off = 0;
+        std::vector<int32_t> tab(tables);
+        int32_t words = 0;
+        std::vector<int32_t> frag_off((size_t)np);
+        for (int k = 0; k < np; ++k) {
+            const int p = dir == 0 ? k : np - 1 - k;
+            const GPhase &gp = phs[(size_t)p];
+            const ItemSet &is = sets[(size_t)p];
+            SplitPhase &D = P.ph[k];
+            D.mode = is.mode;
+            D.B = gp.B;
+            D.B_real = gp.B_real;
+            const int l = is.mode == 0 ? 1 : lm[(size_t)p];
+            const int *jo = gp.B == 16 ? (l == 1 ? joff1_16 : joff2_16) : (l == 1 ? joff1_8 : joff2_8);
+            D.lm = l;
+            D.lane_step = (int32_t)(l * W[(size_t)p]);
+            for (int j = 0; j < 4; ++j) { D.jr[j] = jo[j]; D.j_off[j] = (int32_t)(jo[j] * W[(size_t)p]); }
+            D.items_off = (int32_t)tab.size();
+            D.n_items = (int32_t)is.bases.size();
+            tab.insert(tab.end(), is.bases.begin(), is.bases.end());
+            D.bfrag_off = words;
+            frag_off[(size_t)p] = words;
+            words += (int32_t)(is.block_rel.size() * 32 * (gp.B == 16 ? 4 : 1));
+            // bounds of every address formed from the tables
+            bool ok = true;
+            const int nj = gp.B == 16 ? 4 : 2;
+            for (int32_t b : is.bases) {
+                if (is.mode == 0) ok = ok && b >= 0 && b % 8 == 0 && b + gp.B <= pitch;
+                else
+                    for (int qq = 0; qq < 4; ++qq)
+                        for (int j = 0; j < nj; ++j) {
+                            if (l * qq + jo[j] >= gp.B_real) continue;
+                            const int64_t a = (int64_t)b + (int64_t)qq * D.lane_step + D.j_off[j];
+                            ok = ok && b >= 0 && a % 8 == 0 && a + 8 <= pitch;
+                        }
+            }
+            if (!ok) return HARP_ERR_UNSUPPORTED;
+        }
+        words = (words + 3) / 4 * 4;
+        P.bfrag_words = words;
+        P.tables_len = (int32_t)tab.size();
+        P.tables = upload_s(sp, tab, st);
+        // ---- fragments for every column group
+        std::vector<uint32_t> frag((size_t)n_cg * words, 0u);
+        std::vector<double> F;
+        for (int cgi = 0; cgi < n_cg; ++cgi) {
+            const int64_t cg_base = lower ? (int64_t)cgi * S_mid : (int64_t)cgi * inner;
+            for (int p = 0; p < np; ++p) {
+                const GPhase &gp = phs[(size_t)p];
+                const ItemSet &is = sets[(size_t)p];
+                const int B = gp.B, Br = gp.B_real;
+                const int l = is.mode == 0 ? 1 : lm[(size_t)p];
+                HostPhase hp{gp.t0, gp.t1, Br, gp.S, 0, 1};
+                const int wpl = B == 16 ? 4 : 1;
+                for (size_t bi = 0; bi < is.block_rel.size(); ++bi) {
+                    const int64_t base = cg_base + is.block_rel[bi];
+                    fused_block(plan, hp, base, F);
+                    auto G = [&](int rin, int rout) -> double {
+                        if (rin >= Br || rout >= Br) return 0.0;
+                        double v = dir == 0 ? F[(size_t)rin * Br + rout] : F[(size_t)rout * Br + rin];
+                        if (gp.t0 == 0 && !plan->h_signs.empty()) {
+                            const int64_t pos = base + (int64_t)(dir == 0 ? rin : rout) * gp.S;
+                            v *= (double)plan->h_signs[(size_t)pos];
+                        }
+                        return v;
+                    };
+                    auto slot = [&](int s) { return is.mode == 0 ? s : strided_slot(s, B, l); };
+                    uint32_t *dst0 = frag.data() + (size_t)cgi * words + frag_off[(size_t)p] + bi * 32 * wpl;
+                    for (int lane = 0; lane < 32; ++lane) {
+                        const int gg = lane >> 2, qq = lane & 3;
+                        uint32_t *dst = dst0 + lane * wpl;
+                        if (B == 16) {
+                            for (int nt = 0; nt < 2; ++nt) {
+                                const int n = slot(8 * nt + gg);
+                                dst[2 * nt] = f2bf(G(slot(2 * qq), n)) | ((uint32_t)f2bf(G(slot(2 * qq + 1), n)) << 16);
+                                dst[2 * nt + 1] = f2bf(G(slot(2 * qq + 8), n)) | ((uint32_t)f2bf(G(slot(2 * qq + 9), n)) << 16);
+                            }
+                        } else {
+                            const int n = slot(gg);
+                            dst[0] = f2bf(G(slot(2 * qq), n)) | ((uint32_t)f2bf(G(slot(2 * qq + 1), n)) << 16);
+                        }
+                    }
+                }
+            }
+        }
+        P.bfrag = upload_s(sp, frag, st);
+        const size_t tile_bytes = (size_t)16 * MT * pitch * 2;
+        const size_t need = (tile_bytes + tab.size() * 4 + 15) / 16 * 16 + (size_t)words * 4;
+        ph_out.smem_bytes = std::max(ph_out.smem_bytes, need);
+    }
+    if (st == HARP_OK && ph_out.smem_bytes > 110u * 1024u) return HARP_ERR_UNSUPPORTED;
+    ph_out.present = true;
+    return st;
+}
+
+}  // namespace
+
+harp_status_t harp_split_build(harp_plan *plan) {
+    const int64_t d = plan->d;
+    const int m = plan->st.m;
+    if (d % 8 != 0 || !plan->h_perm.empty()) return HARP_ERR_UNSUPPORTED;
+    // ---- group stages: as many as fit a 16-wide block; smaller products are zero-padded to 8 or 16
+    std::vector<GPhase> phs;
+    for (int t = 0; t < m;) {
+        int64_t prod = 1;
+        int t1 = t;
+        while (t1 < m && prod * plan->st.b[t1] <= 16) prod *= plan->st.b[t1++];
+        if (t1 == t) return HARP_ERR_UNSUPPORTED;                 // a radix above 16
+        phs.push_back({t, t1, prod <= 8 ? 8 : 16, (int)prod, plan->st.s[t]});
+        t = t1;
+    }
+    if (phs[0].B != phs[0].B_real) return HARP_ERR_UNSUPPORTED;   // octets run along the first phase
+    // ---- split point: the longest prefix whose slab has at most 512 coordinates
+    int k = 0;
+    int64_t S_mid = 1;
+    while (k < (int)phs.size() && S_mid * phs[(size_t)k].B_real <= 512) S_mid *= phs[(size_t)k++].B_real;
+    if (k == 0 || S_mid % 8 != 0) return HARP_ERR_UNSUPPORTED;
+    const int64_t U = d / S_mid;
+    std::vector<GPhase> lower(phs.begin(), phs.begin() + k), upper(phs.begin() + k, phs.end());
+    const int Lw = 16;
+    if (!upper.empty() && S_mid % Lw != 0) return HARP_ERR_UNSUPPORTED;
+
+    SplitPlan *sp = new (std::nothrow) SplitPlan();
+    if (!sp) return HARP_ERR_ALLOC;
+    harp_status_t st = build_pass(plan, sp, sp->pass[0], lower, true, S_mid, U, 1);
+    if (st == HARP_OK && !upper.empty()) st = build_pass(plan, sp, sp->pass[1], upper, false, S_mid, U, Lw);
+    if (st == HARP_OK &&
+        cudaFuncSetAttribute(harp_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess)
+        st = HARP_ERR_CUDA;
+    if (st == HARP_OK) {
+        int dev = 0, sms = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (sms > 0) sp->sms = sms;
+        // rows per chunk: both passes of a chunk should find it in L2
+        const char *e = getenv("HARP_SPLIT_CHUNK_MB");
+        const int64_t chunk_bytes = (int64_t)(e ? atoi(e) : 48) << 20;
+        sp->chunk_rows = std::max<int64_t>(64, chunk_bytes / (d * 2) / 64 * 64);
+    }
+    plan->split = sp;
+    if (st != HARP_OK) {
+        cudaGetLastError();
+        harp_split_destroy(plan);
+        return st;
+    }
+    return HARP_OK;
+}
+
+void harp_split_destroy(harp_plan *plan) {
+    if (!plan->split) return;
+    for (void *p : plan->split->dev_allocs) cudaFree(p);
+    delete plan->split;
+    plan->split = nullptr;
+}
+
+harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype, int transpose,
+                               cudaStream_t stream) {
+    const SplitPlan *sp = plan->split;
+    if (!sp || dtype != HARP_BF16) return HARP_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(x) & 15u) != 0) return HARP_ERR_UNSUPPORTED;
+    __nv_bfloat16 *xb = static_cast<__nv_bfloat16 *>(x);
+    const bool two = sp->pass[1].present;
+    for (int64_t r0 = 0; r0 < n_rows; r0 += sp->chunk_rows) {
+        const int64_t r1 = std::min(n_rows, r0 + (two ? sp->chunk_rows : n_rows));
+        for (int s = 0; s < (two ? 2 : 1); ++s) {
+            const int pi = transpose ? (two ? 1 - s : 0) : s;
+            const PassHost &ph = sp->pass[pi];
+            const SplitPass &P = transpose ? ph.bwd : ph.fwd;
+            const int64_t tile_rows = 16 * P.MT;
+            const int64_t n_tiles = (r1 - r0 + tile_rows - 1) / tile_rows;
+            // enough CTAs for a few waves, each keeping its column group for several tiles
+            int64_t parts = std::max<int64_t>(1, ((int64_t)sp->sms * 6 + P.n_cg - 1) / P.n_cg);
+            parts = std::min(parts, n_tiles);
+            const int64_t grid = parts * P.n_cg;
+            harp_split_kernel<<<(unsigned)grid, kSplitThreads, ph.smem_bytes, stream>>>(xb, r0, r1, P);
+            g_harp_launches.fetch_add(1, std::memory_order_relaxed);
+            if (cudaGetLastError() != cudaSuccess) return HARP_ERR_CUDA;
+        }
+        if (!two) break;
+    }
+    return HARP_OK;
+}

@@ -48,3 +48,37 @@ def test_fast_kernel_reports_unsupported(radices, perm, dtype):
     assert st == harp.HARP_ERR_UNSUPPORTED
     harp.apply_(plan, x)                                    # AUTO still works (generic kernel)
     torch.cuda.synchronize()
+
+
+SPLIT = [(4, 4, 4, 4), (8, 8, 8, 8), (16, 16, 8), (2,) * 11, (16, 16, 8, 7), (8, 8, 8, 8, 7), (8, 8, 8, 8, 2),
+         (16, 4, 3, 5), (8, 2, 2, 2, 3), (16, 16, 2, 2, 5)]
+
+
+@pytest.mark.parametrize("radices", SPLIT)
+@pytest.mark.parametrize("kind", ["qr", "identity"])
+def test_split_kernel_matches_oracle(radices, kind):
+    spec = wl.make_plan(29, int(np.prod(radices)), radices, kind, perm="identity", signs=True)
+    oplan = orc.OraclePlan.from_spec(spec)
+    plan = harp.plan_from_spec(spec)
+    rng = np.random.default_rng(9)
+    big = 2100 if spec.d > 10000 else 600            # more rows than one L2 chunk for the wide plans
+    for n_rows in (1, 16, 37, big):
+        xh = host_rows(rng.standard_normal((n_rows, spec.d)), "bf16")
+        x64 = promote(xh, "bf16")
+        for tr in (False, True):
+            got, guards = gpu_apply(plan, xh, "bf16", tr, harp.KERNEL_SPLIT)
+            want = orc.transpose(oplan, x64) if tr else orc.forward(oplan, x64)
+            assert guards
+            if kind == "identity":
+                assert np.array_equal(got, want)
+            else:
+                assert orc.rel_err_rows(got, want) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("radices,perm", [((2,) * 8 + (43,), "identity"), ((4,) * 6, "digit_reversal"), ((7, 2, 4), "identity")])
+def test_split_kernel_reports_unsupported(radices, perm):
+    spec = wl.make_plan(3, int(np.prod(radices)), radices, "qr", perm=perm)
+    plan = harp.plan_from_spec(spec)
+    x = torch.zeros((16, spec.d), device="cuda", dtype=torch.bfloat16)
+    st = harp.lib().harp_apply_ex(plan.handle, x.data_ptr(), 16, 1, 0, harp.KERNEL_SPLIT, None)
+    assert st == harp.HARP_ERR_UNSUPPORTED
