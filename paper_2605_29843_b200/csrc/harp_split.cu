@@ -15,9 +15,10 @@
 // stores out.  Tiles are small, so several CTAs share an SM and their copies overlap with
 // each other's arithmetic.
 //
-// The host walks over the batch in row chunks small enough to stay in L2 and launches
-// pass 1 and pass 2 for a chunk back to back, so that the second pass finds the rows in L2:
-// HBM sees one read and one write per row; only L2 sees two.
+// The host can walk over the batch in row chunks small enough to stay in L2 and launch
+// pass 1 and pass 2 for a chunk back to back, so that the second pass finds the rows in L2
+// (HBM then sees one read and one write per row; only L2 sees two).  See harp_split_build for
+// the default chunk size.
 //
 // Radices that do not fill an 8- or 16-wide block (7, 2, ...) are zero-padded inside the
 // fragments; padded slots read a valid coordinate and are never stored.
@@ -49,7 +50,7 @@ struct SplitPhase {
 };
 
 struct SplitPass {
-    int32_t n_phases, n_cg, n_chunks, pitch, MT;
+    int32_t n_phases, n_cg, n_chunks, pitch, MT, mt_shift;
     int32_t cg_stride;         // global element offset between column groups
     int32_t row_stride;        // d
     int32_t chunk_off;         // tables[chunk_off + 2c] = global offset, [.. + 1] = smem offset of 16-byte chunk c
@@ -66,81 +67,104 @@ __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
     return v;
 }
 
-__global__ void __launch_bounds__(kSplitThreads, 2)
+// B16: the pass has 16-wide phases (more registers, two CTAs per SM); otherwise only 8-wide ones.
+template <bool B16>
+__global__ void __launch_bounds__(kSplitThreads, B16 ? 2 : 3)
 harp_split_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_end, SplitPass P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t sbase = smem_u32(smem_raw);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, q = lane & 3;
-    const int pitch = P.pitch, MT = P.MT;
+    const int pitch = P.pitch, MT = P.MT, mt_shift = P.mt_shift;
     const int tile_rows = 16 * MT;
     const size_t tile_bytes = (size_t)tile_rows * pitch * 2;
     int32_t *tab_s = reinterpret_cast<int32_t *>(smem_raw + tile_bytes);
     const uint32_t bf_s = sbase + (uint32_t)((tile_bytes + (size_t)P.tables_len * 4 + 15) / 16 * 16);
 
     const int cg = blockIdx.x % P.n_cg, part = blockIdx.x / P.n_cg, n_parts = gridDim.x / P.n_cg;
-    // resident data of this column group: tables and fragments
-    for (int i = threadIdx.x; i < P.tables_len; i += kSplitThreads) tab_s[i] = __ldg(P.tables + i);
+    __nv_bfloat16 *xg = x + (size_t)cg * P.cg_stride;
+    const int64_t n_tiles = (row_end - row_begin + tile_rows - 1) / tile_rows;
+    const int64_t rs = P.row_stride;
+
+    // resident data of this column group: fragments (asynchronously; the first tile's wait covers
+    // them) and tables
     {
         const uint32_t *src = P.bfrag + (size_t)cg * P.bfrag_words;
         for (int i = threadIdx.x * 4; i < P.bfrag_words; i += kSplitThreads * 4) cp_async16(bf_s + 4u * i, src + i);
     }
-    cp_async_wait_all();
-    __syncthreads();
+    for (int i = threadIdx.x; i < P.tables_len; i += kSplitThreads) tab_s[i] = __ldg(P.tables + i);
 
-    __nv_bfloat16 *xg = x + (size_t)cg * P.cg_stride;
-    const int64_t n_rows = row_end - row_begin;
-    const int64_t n_tiles = (n_rows + tile_rows - 1) / tile_rows;
-    const int32_t *cmap = tab_s + P.chunk_off;
-    const int64_t rs = P.row_stride;
+    // copy geometry: cp_cols threads share a row and cp_rows rows are copied per step; a thread
+    // keeps the offsets of its (at most four) chunks of a row in registers
+    const int cp_cols = min(P.n_chunks, kSplitThreads), cp_rows = kSplitThreads / cp_cols;
+    const int cp_r = threadIdx.x / cp_cols, cp_c = threadIdx.x - cp_r * cp_cols;
+    const bool copier = cp_r < cp_rows;
+    int32_t goff[4], soff[4];
+#pragma unroll
+    for (int mth = 0; mth < 4; ++mth) {
+        const int ch = cp_c + mth * cp_cols;
+        const bool in = ch < P.n_chunks;
+        goff[mth] = in ? __ldg(P.tables + P.chunk_off + 2 * ch) : -1;
+        soff[mth] = in ? 2 * __ldg(P.tables + P.chunk_off + 2 * ch + 1) : 0;
+    }
 
     for (int64_t tile = part; tile < n_tiles; tile += n_parts) {
         const int64_t row0 = row_begin + tile * tile_rows;
-        const int64_t last = row_end - 1;
         // rows past the end are computed on a copy of the last row and never stored
-        for (int idx = threadIdx.x; idx < tile_rows * P.n_chunks; idx += kSplitThreads) {
-            const int r = idx / P.n_chunks, ch = idx - r * P.n_chunks;
-            const int64_t row = min(row0 + r, last);
-            cp_async16(sbase + 2u * (uint32_t)(r * pitch + cmap[2 * ch + 1]), xg + row * rs + cmap[2 * ch]);
+        if (copier) {
+            const __nv_bfloat16 *last_row = xg + (row_end - 1) * rs;
+            const __nv_bfloat16 *src = xg + (row0 + cp_r) * rs;
+            uint32_t dst = sbase + 2u * (uint32_t)(cp_r * pitch);
+            const int64_t src_step = (int64_t)cp_rows * rs;
+            const uint32_t dst_step = 2u * (uint32_t)(cp_rows * pitch);
+            int64_t row = row0 + cp_r;
+            for (int r = cp_r; r < tile_rows; r += cp_rows, src += src_step, dst += dst_step, row += cp_rows) {
+                const __nv_bfloat16 *s0 = row < row_end ? src : last_row;
+#pragma unroll
+                for (int mth = 0; mth < 4; ++mth)
+                    if (goff[mth] >= 0) cp_async16(dst + soff[mth], s0 + goff[mth]);
+            }
         }
         cp_async_wait_all();
         __syncthreads();
 
         for (int p = 0; p < P.n_phases; ++p) {
             const SplitPhase &ph = P.ph[p];
-            const int n_work = ph.n_items * MT;
             if (ph.mode == 0) {
-                if (ph.B == 16) {
+                // contiguous blocks: one warp takes a block through all row groups of the tile
+                if (B16 && ph.B == 16) {
                     const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
-#pragma unroll 2
-                    for (int w = warp; w < n_work; w += kSplitWarps) {
-                        const int it = w / MT, mt = w - it * MT;
-                        const uint32_t addr = sbase + 2u * (uint32_t)((mt * 16 + mrow) * pitch + tab_s[ph.items_off + it] + mcol);
+                    const uint32_t lane_addr = sbase + 2u * (uint32_t)(mrow * pitch + mcol);
+                    for (int it = warp; it < ph.n_items; it += kSplitWarps) {
                         const uint4 bf = lds128(bf_s + 4u * (uint32_t)(ph.bfrag_off + (it * 32 + lane) * 4));
-                        uint32_t a[4];
-                        ldmatrix_x4(a, addr);
-                        float c0[4], c1[4];
-                        mma_k16(c0, a, bf.x, bf.y);
-                        mma_k16(c1, a, bf.z, bf.w);
-                        stmatrix_x4(addr, pack_bf16(c0[0], c0[1]), pack_bf16(c0[2], c0[3]), pack_bf16(c1[0], c1[1]),
-                                    pack_bf16(c1[2], c1[3]));
+                        uint32_t addr = lane_addr + 2u * (uint32_t)tab_s[ph.items_off + it];
+                        for (int mt = 0; mt < MT; ++mt, addr += 32u * (uint32_t)pitch) {
+                            uint32_t a[4];
+                            ldmatrix_x4(a, addr);
+                            float c0[4], c1[4];
+                            mma_k16(c0, a, bf.x, bf.y);
+                            mma_k16(c1, a, bf.z, bf.w);
+                            stmatrix_x4(addr, pack_bf16(c0[0], c0[1]), pack_bf16(c0[2], c0[3]), pack_bf16(c1[0], c1[1]),
+                                        pack_bf16(c1[2], c1[3]));
+                        }
                     }
                 } else {
-                    const int mrow2 = lane & 15;
-#pragma unroll 2
-                    for (int w = warp; w < n_work; w += kSplitWarps) {
-                        const int it = w / MT, mt = w - it * MT;
-                        const uint32_t addr = sbase + 2u * (uint32_t)((mt * 16 + mrow2) * pitch + tab_s[ph.items_off + it]);
+                    const uint32_t lane_addr = sbase + 2u * (uint32_t)((lane & 15) * pitch);
+                    for (int it = warp; it < ph.n_items; it += kSplitWarps) {
                         const uint32_t bf = lds32(bf_s + 4u * (uint32_t)(ph.bfrag_off + it * 32 + lane));
-                        uint32_t a[2];
-                        ldmatrix_x2(a, addr);
-                        float c0[4];
-                        mma_k8(c0, a, bf);
-                        stmatrix_x2(addr, pack_bf16(c0[0], c0[1]), pack_bf16(c0[2], c0[3]));
+                        uint32_t addr = lane_addr + 2u * (uint32_t)tab_s[ph.items_off + it];
+                        for (int mt = 0; mt < MT; ++mt, addr += 32u * (uint32_t)pitch) {
+                            uint32_t a[2];
+                            ldmatrix_x2(a, addr);
+                            float c0[4];
+                            mma_k8(c0, a, bf);
+                            stmatrix_x2(addr, pack_bf16(c0[0], c0[1]), pack_bf16(c0[2], c0[3]));
+                        }
                     }
                 }
-            } else if (ph.B == 16) {
-                // per-lane slot offsets; padded slots read slot 0 and are not stored
+            } else if (B16 && ph.B == 16) {
+                // strided blocks, eight per item; work unit = (item, row group).  Per-lane slot
+                // offsets: padded slots read slot 0 and are not stored.
                 uint32_t so[4];
                 bool ok[4];
 #pragma unroll
@@ -148,14 +172,16 @@ harp_split_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_
                     ok[j] = ph.lm * q + ph.jr[j] < ph.B_real;
                     so[j] = ok[j] ? 2u * (uint32_t)(q * ph.lane_step + ph.j_off[j]) : 0u;
                 }
+                const int n_work = ph.n_items << mt_shift;
                 for (int w = warp; w < n_work; w += kSplitWarps) {
-                    const int it = w / MT, mt = w - it * MT;
+                    const int it = w >> mt_shift, mt = w & (MT - 1);
                     const uint32_t a0 = sbase + 2u * (uint32_t)((mt * 16 + g) * pitch + tab_s[ph.items_off + it]);
-                    const uint32_t a1 = a0 + 2u * (uint32_t)(8 * pitch);
+                    const uint32_t a1 = a0 + 16u * (uint32_t)pitch;
+                    const uint32_t bfa = bf_s + 4u * (uint32_t)(ph.bfrag_off + (it * 256 + lane) * 4);
                     uint4 raw[4][2], bf[8];
                     uint32_t unused[8][4];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) bf[e] = lds128(bf_s + 4u * (uint32_t)(ph.bfrag_off + ((it * 8 + e) * 32 + lane) * 4));
+                    for (int e = 0; e < 8; ++e) bf[e] = lds128(bfa + e * 512);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         raw[j][0] = lds128(a0 + so[j]);
@@ -178,14 +204,16 @@ harp_split_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_
                     ok[j] = ph.lm * q + ph.jr[j] < ph.B_real;
                     so[j] = ok[j] ? 2u * (uint32_t)(q * ph.lane_step + ph.j_off[j]) : 0u;
                 }
+                const int n_work = ph.n_items << mt_shift;
                 for (int w = warp; w < n_work; w += kSplitWarps) {
-                    const int it = w / MT, mt = w - it * MT;
+                    const int it = w >> mt_shift, mt = w & (MT - 1);
                     const uint32_t a0 = sbase + 2u * (uint32_t)((mt * 16 + g) * pitch + tab_s[ph.items_off + it]);
-                    const uint32_t a1 = a0 + 2u * (uint32_t)(8 * pitch);
+                    const uint32_t a1 = a0 + 16u * (uint32_t)pitch;
+                    const uint32_t bfa = bf_s + 4u * (uint32_t)(ph.bfrag_off + it * 256 + lane);
                     uint4 raw[2][2];
                     uint32_t bf[8];
 #pragma unroll
-                    for (int e = 0; e < 8; ++e) bf[e] = lds32(bf_s + 4u * (uint32_t)(ph.bfrag_off + (it * 8 + e) * 32 + lane));
+                    for (int e = 0; e < 8; ++e) bf[e] = lds32(bfa + e * 128);
 #pragma unroll
                     for (int j = 0; j < 2; ++j) {
                         raw[j][0] = lds128(a0 + so[j]);
@@ -204,15 +232,21 @@ harp_split_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_
             __syncthreads();
         }
 
-        for (int idx = threadIdx.x; idx < tile_rows * P.n_chunks; idx += kSplitThreads) {
-            const int r = idx / P.n_chunks, ch = idx - r * P.n_chunks;
-            if (row0 + r < row_end) {
-                const uint4 v = lds128(sbase + 2u * (uint32_t)(r * pitch + cmap[2 * ch + 1]));
-                stg128(xg + (row0 + r) * rs + cmap[2 * ch], v);
+        if (copier) {
+            __nv_bfloat16 *dstg = xg + (row0 + cp_r) * rs;
+            uint32_t srcs = sbase + 2u * (uint32_t)(cp_r * pitch);
+            const int64_t g_step = (int64_t)cp_rows * rs;
+            const uint32_t s_step = 2u * (uint32_t)(cp_rows * pitch);
+            int64_t row = row0 + cp_r;
+            for (int r = cp_r; r < tile_rows && row < row_end; r += cp_rows, dstg += g_step, srcs += s_step, row += cp_rows) {
+#pragma unroll
+                for (int mth = 0; mth < 4; ++mth)
+                    if (goff[mth] >= 0) stg128(dstg + goff[mth], lds128(srcs + soff[mth]));
             }
         }
         __syncthreads();
     }
+    cp_async_wait_all();      // a CTA without tiles must not exit with copies in flight
 }
 
 // ------------------------------------------------------------------------------- host
@@ -221,6 +255,7 @@ struct PassHost {
     SplitPass fwd{}, bwd{};
     size_t smem_bytes = 0;
     bool present = false;
+    bool has16 = false;
 };
 
 }  // namespace
@@ -290,6 +325,8 @@ harp_status_t build_pass(const harp_plan *plan, SplitPlan *sp, PassHost &ph_out,
     const int n_chunks = lower ? (int)(S_mid / 8) : (int)(U * inner / 8);
     // rows per tile: as many 16-row groups as fit ~40 KB
     int MT = (int)std::max<int64_t>(1, std::min<int64_t>(4, (40 * 1024) / (pitch * 2 * 16)));
+    if (MT == 3) MT = 2;
+    if (n_chunks > 4 * kSplitThreads) return HARP_ERR_UNSUPPORTED;
 
     // ---- tables: chunk map, then items per phase (identical for all column groups and both directions)
     std::vector<int32_t> tables;
@@ -346,6 +383,7 @@ harp_status_t build_pass(const harp_plan *plan, SplitPlan *sp, PassHost &ph_out,
         P.n_chunks = n_chunks;
         P.pitch = (int32_t)pitch;
         P.MT = MT;
+        P.mt_shift = MT == 4 ? 2 : (MT == 2 ? 1 : 0);
         P.cg_stride = lower ? (int32_t)S_mid : inner;
         P.row_stride = (int32_t)d;
         P.chunk_off = 0;
@@ -440,6 +478,7 @@ harp_status_t build_pass(const harp_plan *plan, SplitPlan *sp, PassHost &ph_out,
     }
     if (st == HARP_OK && ph_out.smem_bytes > 110u * 1024u) return HARP_ERR_UNSUPPORTED;
     ph_out.present = true;
+    for (const GPhase &gp : phs) ph_out.has16 = ph_out.has16 || gp.B == 16;
     return st;
 }
 
@@ -475,16 +514,22 @@ harp_status_t harp_split_build(harp_plan *plan) {
     harp_status_t st = build_pass(plan, sp, sp->pass[0], lower, true, S_mid, U, 1);
     if (st == HARP_OK && !upper.empty()) st = build_pass(plan, sp, sp->pass[1], upper, false, S_mid, U, Lw);
     if (st == HARP_OK &&
-        cudaFuncSetAttribute(harp_split_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess)
+        (cudaFuncSetAttribute(harp_split_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess ||
+         cudaFuncSetAttribute(harp_split_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess ||
+         cudaFuncSetAttribute(harp_split_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess ||
+         cudaFuncSetAttribute(harp_split_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess))
         st = HARP_ERR_CUDA;
     if (st == HARP_OK) {
         int dev = 0, sms = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
         if (sms > 0) sp->sms = sms;
-        // rows per chunk: both passes of a chunk should find it in L2
+        // Rows per chunk.  A chunk that fits L2 lets the second pass read what the first wrote
+        // without going to HBM, but every chunk costs two launches and two partial waves; with
+        // the present kernels (bound by instruction issue, not by HBM) large chunks are faster,
+        // so the default is one chunk of up to 8 GiB.  HARP_SPLIT_CHUNK_MB overrides it.
         const char *e = getenv("HARP_SPLIT_CHUNK_MB");
-        const int64_t chunk_bytes = (int64_t)(e ? atoi(e) : 48) << 20;
+        const int64_t chunk_bytes = (int64_t)(e ? atoi(e) : 8192) << 20;
         sp->chunk_rows = std::max<int64_t>(64, chunk_bytes / (d * 2) / 64 * 64);
     }
     plan->split = sp;
@@ -519,10 +564,13 @@ harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, h
             const int64_t tile_rows = 16 * P.MT;
             const int64_t n_tiles = (r1 - r0 + tile_rows - 1) / tile_rows;
             // enough CTAs for a few waves, each keeping its column group for several tiles
-            int64_t parts = std::max<int64_t>(1, ((int64_t)sp->sms * 6 + P.n_cg - 1) / P.n_cg);
+            // one wave of CTAs, each keeping its column group for as many tiles as possible
+            const int per_sm = std::max<int>(1, std::min<int>(ph.has16 ? 2 : 3, (int)((220 * 1024) / (ph.smem_bytes + 1024))));
+            int64_t parts = std::max<int64_t>(1, ((int64_t)sp->sms * per_sm) / P.n_cg);
             parts = std::min(parts, n_tiles);
             const int64_t grid = parts * P.n_cg;
-            harp_split_kernel<<<(unsigned)grid, kSplitThreads, ph.smem_bytes, stream>>>(xb, r0, r1, P);
+            if (ph.has16) harp_split_kernel<true><<<(unsigned)grid, kSplitThreads, ph.smem_bytes, stream>>>(xb, r0, r1, P);
+            else harp_split_kernel<false><<<(unsigned)grid, kSplitThreads, ph.smem_bytes, stream>>>(xb, r0, r1, P);
             g_harp_launches.fetch_add(1, std::memory_order_relaxed);
             if (cudaGetLastError() != cudaSuccess) return HARP_ERR_CUDA;
         }
