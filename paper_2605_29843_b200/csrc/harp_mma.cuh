@@ -46,6 +46,13 @@ __device__ __forceinline__ void mma_k16(float (&c)[4], const uint32_t (&a)[4], u
         : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1), "f"(0.f));
 }
+// D(16x8, fp32) += A(16x16, bf16) . B(16x8, bf16)
+__device__ __forceinline__ void mma_k16_acc(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
 // D(16x8, fp32) = A(16x8, bf16) . B(8x8, bf16)
 __device__ __forceinline__ void mma_k8(float (&c)[4], const uint32_t (&a)[2], uint32_t b0) {
     asm volatile(
@@ -66,6 +73,18 @@ __device__ __forceinline__ uint32_t word_of(const uint4 &v, int w) {
 }
 __device__ __forceinline__ void set_word(uint4 &v, int w, uint32_t x) {
     if (w == 0) v.x = x; else if (w == 1) v.y = x; else if (w == 2) v.z = x; else v.w = x;
+}
+// 8x8 transpose of 16-bit values held as eight uint4 (row i = in[i], eight values each)
+__device__ __forceinline__ void transpose8x8_b16(const uint4 (&in)[8], uint4 (&out)[8]) {
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            const uint32_t x = word_of(in[2 * m], k), y = word_of(in[2 * m + 1], k);
+            set_word(out[2 * k], m, pair_lo(x, y));
+            set_word(out[2 * k + 1], m, pair_hi(x, y));
+        }
+    }
 }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");

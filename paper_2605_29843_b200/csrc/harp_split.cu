@@ -249,6 +249,120 @@ harp_split_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_
     cp_async_wait_all();      // a CTA without tiles must not exit with copies in flight
 }
 
+// ---------------------------------------------------------------------------------------
+// Upper pass with one dense block per position l: all upper stages are fused into a single
+// U x U matrix F_l (U = d / S_mid <= 64, zero-padded to KP = 16*KS).  The tile is stored
+// transposed, [row][l][u], so that a block is KP contiguous values: operands come from
+// ldmatrix, results go back with stmatrix, and the 2-byte transposition is done in registers
+// by the copies (eight 16-byte loads -> 8x8 transpose -> eight 16-byte stores).
+struct UpperPass {
+    int32_t n_cg, Lw, U, KP, NT, pitch, MT;
+    int32_t S_mid, row_stride;
+    const uint32_t *bfrag;     // [column group][l][n-tile][k-step][lane][2]
+    int32_t bfrag_words;
+};
+
+__device__ __forceinline__ uint2 lds64(uint32_t addr) {
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0,%1}, [%2];" : "=r"(v.x), "=r"(v.y) : "r"(addr));
+    return v;
+}
+
+template <int KS>
+__global__ void __launch_bounds__(kSplitThreads, 2)
+harp_upper_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_end, UpperPass P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const uint32_t sbase = smem_u32(smem_raw);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int pitch = P.pitch, MT = P.MT, KP = P.KP, NT = P.NT;
+    const int tile_rows = 16 * MT;
+    const uint32_t bf_s = sbase + (uint32_t)(((size_t)tile_rows * pitch * 2 + 15) / 16 * 16);
+    const int cg = blockIdx.x % P.n_cg, part = blockIdx.x / P.n_cg, n_parts = gridDim.x / P.n_cg;
+    __nv_bfloat16 *xg = x + (size_t)cg * P.Lw;
+    const int64_t n_tiles = (row_end - row_begin + tile_rows - 1) / tile_rows;
+    const int64_t rs = P.row_stride;
+    {
+        const uint32_t *src = P.bfrag + (size_t)cg * P.bfrag_words;
+        for (int i = threadIdx.x * 4; i < P.bfrag_words; i += kSplitThreads * 4) cp_async16(bf_s + 4u * i, src + i);
+    }
+    // copy geometry: a thread owns one (octet of l, octet of u) unit and walks over rows
+    const int lo_n = P.Lw >> 3, uo_n = KP >> 3;
+    const int units_per_row = lo_n * uo_n;
+    const int cp_rows = kSplitThreads / units_per_row;
+    const int cp_r = threadIdx.x / units_per_row, un = threadIdx.x - cp_r * units_per_row;
+    const int uo = un / lo_n, lo = un - uo * lo_n;
+    const int mt_shift = MT == 4 ? 2 : (MT == 2 ? 1 : 0);
+
+    for (int64_t tile = part; tile < n_tiles; tile += n_parts) {
+        const int64_t row0 = row_begin + tile * tile_rows;
+        // ---- copy in, transposing: unit = (row, octet of l, octet of u)
+        for (int r = cp_r; r < tile_rows && cp_r < cp_rows; r += cp_rows) {
+            const int64_t row = min(row0 + r, row_end - 1);
+            const __nv_bfloat16 *src = xg + row * rs + 8 * lo;
+            uint4 in[8], out[8];
+#pragma unroll
+            for (int uu = 0; uu < 8; ++uu) {
+                const int u = 8 * uo + uu;
+                in[uu] = u < P.U ? ldg128_stream(src + (int64_t)u * P.S_mid) : make_uint4(0u, 0u, 0u, 0u);
+            }
+            transpose8x8_b16(in, out);
+            const uint32_t dst = sbase + 2u * (uint32_t)(r * pitch + (8 * lo) * KP + 8 * uo);
+#pragma unroll
+            for (int ll = 0; ll < 8; ++ll) sts128(dst + 2u * (uint32_t)(ll * KP), out[ll]);
+        }
+        cp_async_wait_all();
+        __syncthreads();
+
+        // ---- one dense block per (l, row group)
+        {
+            const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
+            const int n_work = P.Lw * MT;
+            for (int w = warp; w < n_work; w += kSplitWarps) {
+                const int l = w >> mt_shift, mt = w & (MT - 1);
+                const uint32_t addr = sbase + 2u * (uint32_t)((mt * 16 + mrow) * pitch + l * KP + mcol);
+                uint32_t a[KS][4];
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) ldmatrix_x4(a[ks], addr + 32u * ks);
+                const uint32_t bfa = bf_s + 8u * (uint32_t)((l * NT * KS) * 32 + lane);
+                float acc[2 * KS][4];
+#pragma unroll
+                for (int nt = 0; nt < 2 * KS; ++nt) {
+                    acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f;
+                    if (nt < NT) {
+#pragma unroll
+                        for (int ks = 0; ks < KS; ++ks) {
+                            const uint2 b = lds64(bfa + 256u * (uint32_t)(nt * KS + ks));
+                            mma_k16_acc(acc[nt], a[ks], b.x, b.y);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int c = 0; c < KS; ++c)
+                    stmatrix_x4(addr + 32u * c, pack_bf16(acc[2 * c][0], acc[2 * c][1]), pack_bf16(acc[2 * c][2], acc[2 * c][3]),
+                                pack_bf16(acc[2 * c + 1][0], acc[2 * c + 1][1]), pack_bf16(acc[2 * c + 1][2], acc[2 * c + 1][3]));
+            }
+        }
+        __syncthreads();
+
+        // ---- copy out, transposing back
+        for (int r = cp_r; r < tile_rows && cp_r < cp_rows && row0 + r < row_end; r += cp_rows) {
+            const uint32_t srcs = sbase + 2u * (uint32_t)(r * pitch + (8 * lo) * KP + 8 * uo);
+            uint4 in[8], out[8];
+#pragma unroll
+            for (int ll = 0; ll < 8; ++ll) in[ll] = lds128(srcs + 2u * (uint32_t)(ll * KP));
+            transpose8x8_b16(in, out);
+            __nv_bfloat16 *dstg = xg + (row0 + r) * rs + 8 * lo;
+#pragma unroll
+            for (int uu = 0; uu < 8; ++uu) {
+                const int u = 8 * uo + uu;
+                if (u < P.U) stg128(dstg + (int64_t)u * P.S_mid, out[uu]);
+            }
+        }
+        __syncthreads();
+    }
+    cp_async_wait_all();
+}
+
 // ------------------------------------------------------------------------------- host
 
 struct PassHost {
@@ -265,6 +379,11 @@ struct SplitPlan {
     std::vector<void *> dev_allocs;
     int64_t chunk_rows = 0;    // rows per L2-resident chunk
     int sms = 148;
+    // dense upper pass (replaces pass[1] when set)
+    bool dense_upper = false;
+    UpperPass up_fwd{}, up_bwd{};
+    size_t up_smem = 0;
+    int up_ks = 0;
 };
 
 namespace {
@@ -482,23 +601,79 @@ harp_status_t build_pass(const harp_plan *plan, SplitPlan *sp, PassHost &ph_out,
     return st;
 }
 
+
+// All upper stages fused into one U x U block per position l (U <= 64).
+harp_status_t build_dense_upper(const harp_plan *plan, SplitPlan *sp, int t0, int64_t S_mid, int64_t U) {
+    if (U > 64 || U < 2) return HARP_ERR_UNSUPPORTED;
+    const int KP = (int)((U + 15) / 16 * 16), KS = KP / 16, NT = (int)((U + 7) / 8);
+    const int64_t per_l_words = (int64_t)NT * KS * 64;
+    int Lw = 16;
+    if (S_mid % 16 != 0 || 16 * per_l_words * 4 > 80 * 1024) Lw = 8;
+    if (S_mid % Lw != 0) return HARP_ERR_UNSUPPORTED;
+    int64_t pitch = (int64_t)Lw * KP;
+    if ((pitch / 8) % 2 == 0) pitch += 8;
+    const int64_t frag_bytes = Lw * per_l_words * 4;
+    int MT = 1;
+    while (MT < 4 && (int64_t)32 * MT * pitch * 2 + frag_bytes <= 100 * 1024) MT *= 2;
+    const size_t smem = ((size_t)16 * MT * pitch * 2 + 15) / 16 * 16 + (size_t)frag_bytes;
+    if (smem > 110u * 1024u) return HARP_ERR_UNSUPPORTED;
+    if ((Lw / 8) * (KP / 8) > kSplitThreads) return HARP_ERR_UNSUPPORTED;
+    const int n_cg = (int)(S_mid / Lw);
+    harp_status_t st = HARP_OK;
+    HostPhase hp{t0, plan->st.m, (int)U, S_mid, 0, 1};
+    std::vector<double> F;
+    for (int dir = 0; dir < 2 && st == HARP_OK; ++dir) {
+        UpperPass &P = dir == 0 ? sp->up_fwd : sp->up_bwd;
+        P.n_cg = n_cg; P.Lw = Lw; P.U = (int32_t)U; P.KP = KP; P.NT = NT; P.pitch = (int32_t)pitch; P.MT = MT;
+        P.S_mid = (int32_t)S_mid; P.row_stride = (int32_t)plan->d;
+        P.bfrag_words = (int32_t)(Lw * per_l_words);
+        std::vector<uint32_t> frag((size_t)n_cg * P.bfrag_words, 0u);
+        for (int cgi = 0; cgi < n_cg; ++cgi)
+            for (int l = 0; l < Lw; ++l) {
+                const int64_t base = (int64_t)cgi * Lw + l;
+                fused_block(plan, hp, base, F);
+                auto G = [&](int rin, int rout) -> double {
+                    if (rin >= U || rout >= U) return 0.0;
+                    return dir == 0 ? F[(size_t)rin * U + rout] : F[(size_t)rout * U + rin];
+                };
+                uint32_t *dst0 = frag.data() + (size_t)cgi * P.bfrag_words + (size_t)l * per_l_words;
+                for (int nt = 0; nt < NT; ++nt)
+                    for (int ks = 0; ks < KS; ++ks)
+                        for (int lane = 0; lane < 32; ++lane) {
+                            const int gg = lane >> 2, qq = lane & 3;
+                            const int n = 8 * nt + gg, k0 = 16 * ks + 2 * qq;
+                            uint32_t *dst = dst0 + ((size_t)(nt * KS + ks) * 32 + lane) * 2;
+                            dst[0] = f2bf(G(k0, n)) | ((uint32_t)f2bf(G(k0 + 1, n)) << 16);
+                            dst[1] = f2bf(G(k0 + 8, n)) | ((uint32_t)f2bf(G(k0 + 9, n)) << 16);
+                        }
+            }
+        P.bfrag = upload_s(sp, frag, st);
+    }
+    sp->dense_upper = true;
+    sp->up_smem = smem;
+    sp->up_ks = KS;
+    return st;
+}
+
 }  // namespace
 
 harp_status_t harp_split_build(harp_plan *plan) {
     const int64_t d = plan->d;
     const int m = plan->st.m;
     if (d % 8 != 0 || !plan->h_perm.empty()) return HARP_ERR_UNSUPPORTED;
-    // ---- group stages: as many as fit a 16-wide block; smaller products are zero-padded to 8 or 16
+    // ---- group stages: as many as fit a 16-wide block; smaller products are zero-padded to 8 or 16.
+    // A radix above 16 ends the grouping: it and everything after it form the dense upper block.
     std::vector<GPhase> phs;
+    int t_big = m;
     for (int t = 0; t < m;) {
+        if (plan->st.b[t] > 16) { t_big = t; break; }
         int64_t prod = 1;
         int t1 = t;
         while (t1 < m && prod * plan->st.b[t1] <= 16) prod *= plan->st.b[t1++];
-        if (t1 == t) return HARP_ERR_UNSUPPORTED;                 // a radix above 16
         phs.push_back({t, t1, prod <= 8 ? 8 : 16, (int)prod, plan->st.s[t]});
         t = t1;
     }
-    if (phs[0].B != phs[0].B_real) return HARP_ERR_UNSUPPORTED;   // octets run along the first phase
+    if (phs.empty() || phs[0].B != phs[0].B_real) return HARP_ERR_UNSUPPORTED;   // octets run along the first phase
     // ---- split point: the longest prefix whose slab has at most 512 coordinates
     int k = 0;
     int64_t S_mid = 1;
@@ -507,17 +682,24 @@ harp_status_t harp_split_build(harp_plan *plan) {
     const int64_t U = d / S_mid;
     std::vector<GPhase> lower(phs.begin(), phs.begin() + k), upper(phs.begin() + k, phs.end());
     const int Lw = 16;
-    if (!upper.empty() && S_mid % Lw != 0) return HARP_ERR_UNSUPPORTED;
+    const bool want_dense = t_big < m || (getenv("HARP_UPPER_DENSE") && atoi(getenv("HARP_UPPER_DENSE")) && U > 1);
+    if (t_big < m && k != (int)phs.size()) return HARP_ERR_UNSUPPORTED;            // big radix must follow the slab directly
+    if (!want_dense && !upper.empty() && S_mid % Lw != 0) return HARP_ERR_UNSUPPORTED;
 
     SplitPlan *sp = new (std::nothrow) SplitPlan();
     if (!sp) return HARP_ERR_ALLOC;
     harp_status_t st = build_pass(plan, sp, sp->pass[0], lower, true, S_mid, U, 1);
-    if (st == HARP_OK && !upper.empty()) st = build_pass(plan, sp, sp->pass[1], upper, false, S_mid, U, Lw);
+    if (st == HARP_OK && want_dense) st = build_dense_upper(plan, sp, lower.back().t1, S_mid, U);
+    else if (st == HARP_OK && !upper.empty()) st = build_pass(plan, sp, sp->pass[1], upper, false, S_mid, U, Lw);
     if (st == HARP_OK &&
         (cudaFuncSetAttribute(harp_split_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess ||
          cudaFuncSetAttribute(harp_split_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess ||
          cudaFuncSetAttribute(harp_split_kernel<true>, cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess ||
-         cudaFuncSetAttribute(harp_split_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess))
+         cudaFuncSetAttribute(harp_split_kernel<false>, cudaFuncAttributePreferredSharedMemoryCarveout, 100) != cudaSuccess ||
+         cudaFuncSetAttribute(harp_upper_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess ||
+         cudaFuncSetAttribute(harp_upper_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess ||
+         cudaFuncSetAttribute(harp_upper_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess ||
+         cudaFuncSetAttribute(harp_upper_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess))
         st = HARP_ERR_CUDA;
     if (st == HARP_OK) {
         int dev = 0, sms = 0;
@@ -554,16 +736,33 @@ harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, h
     if (!sp || dtype != HARP_BF16) return HARP_ERR_UNSUPPORTED;
     if ((reinterpret_cast<uintptr_t>(x) & 15u) != 0) return HARP_ERR_UNSUPPORTED;
     __nv_bfloat16 *xb = static_cast<__nv_bfloat16 *>(x);
-    const bool two = sp->pass[1].present;
+    const bool two = sp->pass[1].present || sp->dense_upper;
     for (int64_t r0 = 0; r0 < n_rows; r0 += sp->chunk_rows) {
         const int64_t r1 = std::min(n_rows, r0 + (two ? sp->chunk_rows : n_rows));
         for (int s = 0; s < (two ? 2 : 1); ++s) {
             const int pi = transpose ? (two ? 1 - s : 0) : s;
+            if (pi == 1 && sp->dense_upper) {
+                const UpperPass &P = transpose ? sp->up_bwd : sp->up_fwd;
+                const int64_t tile_rows = 16 * P.MT;
+                const int64_t n_tiles = (r1 - r0 + tile_rows - 1) / tile_rows;
+                const int per_sm = std::max<int>(1, std::min<int>(2, (int)((220 * 1024) / (sp->up_smem + 1024))));
+                int64_t parts = std::max<int64_t>(1, ((int64_t)sp->sms * per_sm) / P.n_cg);
+                parts = std::min(parts, n_tiles);
+                const unsigned grid = (unsigned)(parts * P.n_cg);
+                switch (sp->up_ks) {
+                    case 1: harp_upper_kernel<1><<<grid, kSplitThreads, sp->up_smem, stream>>>(xb, r0, r1, P); break;
+                    case 2: harp_upper_kernel<2><<<grid, kSplitThreads, sp->up_smem, stream>>>(xb, r0, r1, P); break;
+                    case 3: harp_upper_kernel<3><<<grid, kSplitThreads, sp->up_smem, stream>>>(xb, r0, r1, P); break;
+                    default: harp_upper_kernel<4><<<grid, kSplitThreads, sp->up_smem, stream>>>(xb, r0, r1, P); break;
+                }
+                g_harp_launches.fetch_add(1, std::memory_order_relaxed);
+                if (cudaGetLastError() != cudaSuccess) return HARP_ERR_CUDA;
+                continue;
+            }
             const PassHost &ph = sp->pass[pi];
             const SplitPass &P = transpose ? ph.bwd : ph.fwd;
             const int64_t tile_rows = 16 * P.MT;
             const int64_t n_tiles = (r1 - r0 + tile_rows - 1) / tile_rows;
-            // enough CTAs for a few waves, each keeping its column group for several tiles
             // one wave of CTAs, each keeping its column group for as many tiles as possible
             const int per_sm = std::max<int>(1, std::min<int>(ph.has16 ? 2 : 3, (int)((220 * 1024) / (ph.smem_bytes + 1024))));
             int64_t parts = std::max<int64_t>(1, ((int64_t)sp->sms * per_sm) / P.n_cg);

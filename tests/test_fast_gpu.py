@@ -51,7 +51,8 @@ def test_fast_kernel_reports_unsupported(radices, perm, dtype):
 
 
 SPLIT = [(4, 4, 4, 4), (8, 8, 8, 8), (16, 16, 8), (2,) * 11, (16, 16, 8, 7), (8, 8, 8, 8, 7), (8, 8, 8, 8, 2),
-         (16, 4, 3, 5), (8, 2, 2, 2, 3), (16, 16, 2, 2, 5)]
+         (16, 4, 3, 5), (8, 2, 2, 2, 3), (16, 16, 2, 2, 5), (2,) * 8 + (43,), (16, 16, 17), (8, 8, 8, 33),
+         (4, 4, 4, 4, 64), (8, 8, 21, 3)]
 
 
 @pytest.mark.parametrize("radices", SPLIT)
@@ -75,7 +76,23 @@ def test_split_kernel_matches_oracle(radices, kind):
                 assert orc.rel_err_rows(got, want) <= TOL["bf16"]
 
 
-@pytest.mark.parametrize("radices,perm", [((2,) * 8 + (43,), "identity"), ((4,) * 6, "digit_reversal"), ((7, 2, 4), "identity")])
+@pytest.mark.parametrize("radices", [(16, 16, 8, 7), (8, 8, 8, 8, 7), (8, 8, 8, 8)])
+def test_split_kernel_with_dense_upper_block(radices, monkeypatch):
+    monkeypatch.setenv("HARP_UPPER_DENSE", "1")
+    spec = wl.make_plan(31, int(np.prod(radices)), radices, "qr", perm="identity", signs=True)
+    oplan = orc.OraclePlan.from_spec(spec)
+    plan = harp.plan_from_spec(spec)
+    rng = np.random.default_rng(10)
+    for n_rows in (5, 100):
+        xh = host_rows(rng.standard_normal((n_rows, spec.d)), "bf16")
+        x64 = promote(xh, "bf16")
+        for tr in (False, True):
+            got, guards = gpu_apply(plan, xh, "bf16", tr, harp.KERNEL_SPLIT)
+            want = orc.transpose(oplan, x64) if tr else orc.forward(oplan, x64)
+            assert guards and orc.rel_err_rows(got, want) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("radices,perm", [((2,) * 8 + (67,), "identity"), ((4,) * 6, "digit_reversal"), ((7, 2, 4), "identity")])
 def test_split_kernel_reports_unsupported(radices, perm):
     spec = wl.make_plan(3, int(np.prod(radices)), radices, "qr", perm=perm)
     plan = harp.plan_from_spec(spec)
