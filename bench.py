@@ -33,9 +33,10 @@ METRIC = "harp_apply_rows_per_s"
 UNIT = "rows/s"
 WORKLOAD = "cfg2: d=4096 radix-4 x6, signs + digit-reversal perm, 16384 rows bf16, forward+transpose per step"
 N_BUF = 4
-# DRAM bytes (read+write) per launch of the dominant kernel on the headline workload,
-# from the ncu capture summarised in profiles/ (None until captured).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of harp_fast_kernel on the
+# headline workload, mean of the forward and the transpose launch in profiles/harp_fast_kernel_cfg2.md
+# (read 134.9 / 134.8 MB, write 101.4 / 88.3 MB: the last tiles' write-back is still in L2 at kernel end).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 229_650_000
 
 
 def measured_peaks():
@@ -248,7 +249,8 @@ def run_gpu(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     harp.lib()
-    kernel = {"auto": harp.KERNEL_AUTO, "generic": harp.KERNEL_GENERIC, "fast": harp.KERNEL_FAST}[args.kernel]
+    kernel = {"auto": harp.KERNEL_AUTO, "generic": harp.KERNEL_GENERIC, "fast": harp.KERNEL_FAST,
+              "split": harp.KERNEL_SPLIT}[args.kernel]
 
     w = wl.config(2)
     spec, data = w.plans["q"], w.data["x"]
@@ -341,18 +343,44 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def run_profile_case(args):
+    """Small case for profilers: `--profile-config C` applies configuration C's processor to
+    `--profile-rows` seeded device rows, alternating forward and transpose, `--profile-reps` times."""
+    import torch
+    import paper_2605_29843_b200 as harp
+    kernel = {"auto": harp.KERNEL_AUTO, "generic": harp.KERNEL_GENERIC, "fast": harp.KERNEL_FAST,
+              "split": harp.KERNEL_SPLIT}[args.kernel]
+    w = wl.config(args.profile_config)
+    spec = w.plans["in"] if args.profile_config == 5 else w.plans["q"]
+    plan = harp.plan_from_spec(spec)
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(7)
+    tdt = torch.float32 if w.data["x"].dtype == "f32" else torch.bfloat16
+    x = torch.randn((args.profile_rows, spec.d), generator=gen, device="cuda").to(tdt)
+    for i in range(args.profile_reps):
+        harp.apply_(plan, x, transpose=bool(i & 1), kernel=kernel)
+    torch.cuda.synchronize()
+    print(json.dumps({"profile_case": w.name, "rows": args.profile_rows, "reps": args.profile_reps,
+                      "launches": harp.harp_launch_count()}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="harp", choices=["harp", "reference"])
-    ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "fast"])
+    ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "fast", "split"])
+    ap.add_argument("--profile-config", type=int, default=0, help="run a small profiling case of this configuration and exit")
+    ap.add_argument("--profile-rows", type=int, default=8192)
+    ap.add_argument("--profile-reps", type=int, default=2)
     ap.add_argument("--all-configs", action="store_true")
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU-oracle baseline")
     ap.add_argument("--ref-rows", type=int, default=2048)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.profile_config:
+        run_profile_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)

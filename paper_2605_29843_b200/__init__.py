@@ -164,6 +164,14 @@ def harp_apply_host(plan: Plan, host_ptr: int, n_rows: int, dtype: int, transpos
         raise HarpError(st, "harp_apply_host")
 
 
+def shard_rows(n_rows: int, rank: int, world: int):
+    """Contiguous row range [start, stop) of `rank` when a batch is split over `world` ranks.
+    Rows are independent, so ranks need no collective on the data path."""
+    base, rem = divmod(int(n_rows), int(world))
+    start = rank * base + min(rank, rem)
+    return start, start + base + (1 if rank < rem else 0)
+
+
 # ---- torch conveniences (device memory and streams only) ----
 
 def _torch_dtype_code(t) -> int:

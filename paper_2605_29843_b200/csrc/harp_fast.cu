@@ -157,12 +157,16 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
         c.xB = x + min(row0 + c.g + 8, last) * d;
 
         if (P.copy_in >= 0) {
+            // a thread owns the same 16-byte chunks of every row; no index arithmetic per chunk
             const int32_t *cmap = tab_s + P.copy_in;
             const int chunks = d >> 3;
-            for (int idx = threadIdx.x; idx < kTileRows * chunks; idx += NT) {
-                const int r = idx / chunks, ch = idx - r * chunks;
-                const int64_t row = min(row0 + r, last);
-                cp_async16(c.sbase + 2u * (uint32_t)(r * pitch + cmap[ch]), x + row * d + 8 * ch);
+            for (int ch = threadIdx.x; ch < chunks; ch += NT) {
+                const uint32_t dst = c.sbase + 2u * (uint32_t)cmap[ch];
+                const __nv_bfloat16 *src = x + row0 * d + 8 * ch;
+                const __nv_bfloat16 *last_src = x + last * d + 8 * ch;
+#pragma unroll 4
+                for (int r = 0; r < kTileRows; ++r)
+                    cp_async16(dst + 2u * (uint32_t)(r * pitch), row0 + r <= last ? src + (int64_t)r * d : last_src);
             }
             cp_async_wait_all();
             __syncthreads();
@@ -430,12 +434,12 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
         if (P.copy_out >= 0) {
             const int32_t *cmap = tab_s + P.copy_out;
             const int chunks = d >> 3;
-            for (int idx = threadIdx.x; idx < kTileRows * chunks; idx += NT) {
-                const int r = idx / chunks, ch = idx - r * chunks;
-                if (row0 + r < n_rows) {
-                    const uint4 v = lds128(c.sbase + 2u * (uint32_t)(r * pitch + cmap[ch]));
-                    stg128(x + (row0 + r) * d + 8 * ch, v);
-                }
+            const int rows = (int)min((int64_t)kTileRows, n_rows - row0);
+            for (int ch = threadIdx.x; ch < chunks; ch += NT) {
+                const uint32_t src = c.sbase + 2u * (uint32_t)cmap[ch];
+                __nv_bfloat16 *dst = x + row0 * d + 8 * ch;
+#pragma unroll 4
+                for (int r = 0; r < rows; ++r) stg128(dst + (int64_t)r * d, lds128(src + 2u * (uint32_t)(r * pitch)));
             }
             __syncthreads();
         }
