@@ -51,6 +51,7 @@ struct SplitPhase {
 
 struct SplitPass {
     int32_t n_phases, n_cg, n_chunks, pitch, MT, mt_shift;
+    int32_t n_buf;             // 2: the next tile is copied in while this one is multiplied; 1: single buffer
     int32_t cg_stride;         // global element offset between column groups
     int32_t row_stride;        // d
     int32_t chunk_off;         // tables[chunk_off + 2c] = global offset, [.. + 1] = smem offset of 16-byte chunk c
@@ -72,14 +73,15 @@ template <bool B16>
 __global__ void __launch_bounds__(kSplitThreads, B16 ? 2 : 3)
 harp_split_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_end, SplitPass P) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    const uint32_t sbase = smem_u32(smem_raw);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, q = lane & 3;
     const int pitch = P.pitch, MT = P.MT, mt_shift = P.mt_shift;
     const int tile_rows = 16 * MT;
-    const size_t tile_bytes = (size_t)tile_rows * pitch * 2;
-    int32_t *tab_s = reinterpret_cast<int32_t *>(smem_raw + tile_bytes);
-    const uint32_t bf_s = sbase + (uint32_t)((tile_bytes + (size_t)P.tables_len * 4 + 15) / 16 * 16);
+    const size_t tile_bytes = (size_t)tile_rows * pitch * 2;          // a multiple of 16
+    const uint32_t sbase0 = smem_u32(smem_raw);                        // tile buffer(s), then tables, then fragments
+    const int n_buf = P.n_buf;
+    int32_t *tab_s = reinterpret_cast<int32_t *>(smem_raw + n_buf * tile_bytes);
+    const uint32_t bf_s = sbase0 + (uint32_t)((n_buf * tile_bytes + (size_t)P.tables_len * 4 + 15) / 16 * 16);
 
     const int cg = blockIdx.x % P.n_cg, part = blockIdx.x / P.n_cg, n_parts = gridDim.x / P.n_cg;
     __nv_bfloat16 *xg = x + (size_t)cg * P.cg_stride;
@@ -99,6 +101,7 @@ harp_split_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_
     const int cp_cols = min(P.n_chunks, kSplitThreads), cp_rows = kSplitThreads / cp_cols;
     const int cp_r = threadIdx.x / cp_cols, cp_c = threadIdx.x - cp_r * cp_cols;
     const bool copier = cp_r < cp_rows;
+    const bool single_chunk = P.n_chunks <= kSplitThreads;
     int32_t goff[4], soff[4];
 #pragma unroll
     for (int mth = 0; mth < 4; ++mth) {
@@ -108,24 +111,55 @@ harp_split_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_
         soff[mth] = in ? 2 * __ldg(P.tables + P.chunk_off + 2 * ch + 1) : 0;
     }
 
-    for (int64_t tile = part; tile < n_tiles; tile += n_parts) {
+    // With two buffers the copy of the next tile is in flight while this one is multiplied; passes
+    // whose occupancy is limited by shared memory rather than registers use one buffer instead.
+    auto copy_in = [&](int64_t tile, uint32_t sb) {
         const int64_t row0 = row_begin + tile * tile_rows;
         // rows past the end are computed on a copy of the last row and never stored
         if (copier) {
-            const __nv_bfloat16 *last_row = xg + (row_end - 1) * rs;
-            const __nv_bfloat16 *src = xg + (row0 + cp_r) * rs;
-            uint32_t dst = sbase + 2u * (uint32_t)(cp_r * pitch);
-            const int64_t src_step = (int64_t)cp_rows * rs;
-            const uint32_t dst_step = 2u * (uint32_t)(cp_rows * pitch);
-            int64_t row = row0 + cp_r;
-            for (int r = cp_r; r < tile_rows; r += cp_rows, src += src_step, dst += dst_step, row += cp_rows) {
-                const __nv_bfloat16 *s0 = row < row_end ? src : last_row;
+            if (row0 + tile_rows <= row_end && single_chunk) {
+                const __nv_bfloat16 *src = xg + (row0 + cp_r) * rs + goff[0];
+                uint32_t dst = sb + 2u * (uint32_t)(cp_r * pitch) + soff[0];
+                const int64_t src_step = (int64_t)cp_rows * rs;
+                const uint32_t dst_step = 2u * (uint32_t)(cp_rows * pitch);
+#pragma unroll 4
+                for (int r = cp_r; r < tile_rows; r += cp_rows, src += src_step, dst += dst_step) cp_async16(dst, src);
+            } else {
+                const __nv_bfloat16 *last_row = xg + (row_end - 1) * rs;
+                const __nv_bfloat16 *src = xg + (row0 + cp_r) * rs;
+                uint32_t dst = sb + 2u * (uint32_t)(cp_r * pitch);
+                const int64_t src_step = (int64_t)cp_rows * rs;
+                const uint32_t dst_step = 2u * (uint32_t)(cp_rows * pitch);
+                int64_t row = row0 + cp_r;
+                for (int r = cp_r; r < tile_rows; r += cp_rows, src += src_step, dst += dst_step, row += cp_rows) {
+                    const __nv_bfloat16 *s0 = row < row_end ? src : last_row;
 #pragma unroll
-                for (int mth = 0; mth < 4; ++mth)
-                    if (goff[mth] >= 0) cp_async16(dst + soff[mth], s0 + goff[mth]);
+                    for (int mth = 0; mth < 4; ++mth)
+                        if (goff[mth] >= 0) cp_async16(dst + soff[mth], s0 + goff[mth]);
+                }
             }
         }
-        cp_async_wait_all();
+        cp_async_commit();
+    };
+
+    int buf = 0;
+    if (n_buf == 2 && part < n_tiles) copy_in(part, sbase0);
+    for (int64_t tile = part; tile < n_tiles; tile += n_parts) {
+        const int64_t row0 = row_begin + tile * tile_rows;
+        const bool full_tile = row0 + tile_rows <= row_end;
+        const uint32_t sbase = sbase0 + (uint32_t)(buf * tile_bytes);
+        if (n_buf == 2) {
+            if (tile + n_parts < n_tiles) {
+                copy_in(tile + n_parts, sbase0 + (uint32_t)((buf ^ 1) * tile_bytes));
+                cp_async_wait_group<1>();
+            } else {
+                cp_async_wait_group<0>();
+            }
+            buf ^= 1;
+        } else {
+            copy_in(tile, sbase0);
+            cp_async_wait_group<0>();
+        }
         __syncthreads();
 
         for (int p = 0; p < P.n_phases; ++p) {
@@ -233,15 +267,24 @@ harp_split_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_
         }
 
         if (copier) {
-            __nv_bfloat16 *dstg = xg + (row0 + cp_r) * rs;
-            uint32_t srcs = sbase + 2u * (uint32_t)(cp_r * pitch);
-            const int64_t g_step = (int64_t)cp_rows * rs;
-            const uint32_t s_step = 2u * (uint32_t)(cp_rows * pitch);
-            int64_t row = row0 + cp_r;
-            for (int r = cp_r; r < tile_rows && row < row_end; r += cp_rows, dstg += g_step, srcs += s_step, row += cp_rows) {
+            if (full_tile && single_chunk) {
+                __nv_bfloat16 *dstg = xg + (row0 + cp_r) * rs + goff[0];
+                uint32_t srcs = sbase + 2u * (uint32_t)(cp_r * pitch) + soff[0];
+                const int64_t g_step = (int64_t)cp_rows * rs;
+                const uint32_t s_step = 2u * (uint32_t)(cp_rows * pitch);
+#pragma unroll 4
+                for (int r = cp_r; r < tile_rows; r += cp_rows, dstg += g_step, srcs += s_step) stg128(dstg, lds128(srcs));
+            } else {
+                __nv_bfloat16 *dstg = xg + (row0 + cp_r) * rs;
+                uint32_t srcs = sbase + 2u * (uint32_t)(cp_r * pitch);
+                const int64_t g_step = (int64_t)cp_rows * rs;
+                const uint32_t s_step = 2u * (uint32_t)(cp_rows * pitch);
+                int64_t row = row0 + cp_r;
+                for (int r = cp_r; r < tile_rows && row < row_end; r += cp_rows, dstg += g_step, srcs += s_step, row += cp_rows) {
 #pragma unroll
-                for (int mth = 0; mth < 4; ++mth)
-                    if (goff[mth] >= 0) stg128(dstg + goff[mth], lds128(srcs + soff[mth]));
+                    for (int mth = 0; mth < 4; ++mth)
+                        if (goff[mth] >= 0) stg128(dstg + goff[mth], lds128(srcs + soff[mth]));
+                }
             }
         }
         __syncthreads();
@@ -592,7 +635,11 @@ harp_status_t build_pass(const harp_plan *plan, SplitPlan *sp, PassHost &ph_out,
         }
         P.bfrag = upload_s(sp, frag, st);
         const size_t tile_bytes = (size_t)16 * MT * pitch * 2;
-        const size_t need = (tile_bytes + tab.size() * 4 + 15) / 16 * 16 + (size_t)words * 4;
+        bool any16 = false;
+        for (const GPhase &gp : phs) any16 = any16 || gp.B == 16;
+        const size_t one = (tile_bytes + tab.size() * 4 + 15) / 16 * 16 + (size_t)words * 4;
+        P.n_buf = (any16 && one + tile_bytes <= 100u * 1024u) ? 2 : 1;
+        const size_t need = (P.n_buf * tile_bytes + tab.size() * 4 + 15) / 16 * 16 + (size_t)words * 4;
         ph_out.smem_bytes = std::max(ph_out.smem_bytes, need);
     }
     if (st == HARP_OK && ph_out.smem_bytes > 110u * 1024u) return HARP_ERR_UNSUPPORTED;
