@@ -8,6 +8,8 @@
 // This path defines correct behaviour for every plan the ABI accepts (up to the
 // shared-memory capacity); the tensor-core path in harp_fast.cu is faster where
 // it applies.
+#include <algorithm>
+
 #include "harp_internal.h"
 
 namespace {
@@ -97,6 +99,109 @@ harp_generic_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_cta, 
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Block-owner kernel (radices up to 8): a thread owns one block of the current stage, keeps its
+// b x b kernel in registers and walks over the rows of the tile, so a block kernel is fetched
+// once per tile instead of once per output coordinate, all index arithmetic is done once per
+// block, and (a block being updated in place by its only owner) one barrier per stage suffices.
+template <int B>
+__device__ __forceinline__ void stage_blocks(float *v, int rows, int d, int s, const float *__restrict__ Kt, int transpose) {
+    const int nblk = d / B;
+    for (int c = threadIdx.x; c < nblk; c += blockDim.x) {
+        const int alpha = c / s, beta = c - alpha * s;
+        float *p = v + alpha * B * s + beta;
+        float K[B][B];
+        const float *Kc = Kt + (size_t)c * B * B;
+        // a stage's block array starts at a multiple of 4 bytes only; the 16-byte load needs more
+        if (B == 2 && (reinterpret_cast<uintptr_t>(Kt) & 15u) == 0) {
+            const float4 k4 = __ldg(reinterpret_cast<const float4 *>(Kc));
+            K[0][0] = k4.x;
+            K[0][1] = transpose ? k4.z : k4.y;
+            K[1][0] = transpose ? k4.y : k4.z;
+            K[1][1] = k4.w;
+        } else {
+#pragma unroll
+            for (int i = 0; i < B; ++i)
+#pragma unroll
+                for (int j = 0; j < B; ++j) K[i][j] = __ldg(Kc + (transpose ? j * B + i : i * B + j));
+        }
+#pragma unroll 2
+        for (int r = 0; r < rows; ++r, p += d) {
+            float in[B];
+#pragma unroll
+            for (int i = 0; i < B; ++i) in[i] = p[i * s];
+#pragma unroll
+            for (int j = 0; j < B; ++j) {
+                float a = in[0] * K[0][j];
+#pragma unroll
+                for (int i = 1; i < B; ++i) a = fmaf(in[i], K[i][j], a);
+                p[j * s] = a;
+            }
+        }
+    }
+}
+
+template <typename T, int NT, bool BIG>
+__global__ void __launch_bounds__(NT, 1)
+harp_blockowner_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_cta, StageTable st,
+                       const float *__restrict__ blocks, const int32_t *__restrict__ perm,
+                       const int8_t *__restrict__ signs, int transpose) {
+    extern __shared__ float v[];                     // [rows_per_cta][d]
+    const int64_t row0 = (int64_t)blockIdx.x * rows_per_cta;
+    const int rows = (int)min((int64_t)rows_per_cta, n_rows - row0);
+    T *xt = x + row0 * d;
+    // a1-a3: load, sign, gather (forward) -- or plain load (transpose); a thread keeps its columns
+    for (int i = threadIdx.x; i < d; i += NT) {
+        const int src = (!transpose && perm) ? perm[i] : i;
+        const float sg = (!transpose && signs && signs[src] < 0) ? -1.f : 1.f;
+        const T *col = xt + src;
+        for (int r = 0; r < rows; ++r) v[r * d + i] = sg * to_f32<T>(col[(int64_t)r * d]);
+    }
+    __syncthreads();
+    for (int k = 0; k < st.m; ++k) {
+        const int t = transpose ? st.m - 1 - k : k;
+        const float *Kt = blocks + st.off[t];
+        const int b = st.b[t];
+        if (b == 2) stage_blocks<2>(v, rows, d, st.s[t], Kt, transpose);
+        else if (b == 3) stage_blocks<3>(v, rows, d, st.s[t], Kt, transpose);
+        else if (b == 4) stage_blocks<4>(v, rows, d, st.s[t], Kt, transpose);
+        else if (BIG) {
+            if (b == 5) stage_blocks<5>(v, rows, d, st.s[t], Kt, transpose);
+            else if (b == 6) stage_blocks<6>(v, rows, d, st.s[t], Kt, transpose);
+            else if (b == 7) stage_blocks<7>(v, rows, d, st.s[t], Kt, transpose);
+            else stage_blocks<8>(v, rows, d, st.s[t], Kt, transpose);
+        }
+        __syncthreads();
+    }
+    // a5: store -- or scatter and sign (transpose)
+    for (int i = threadIdx.x; i < d; i += NT) {
+        const int dst = (transpose && perm) ? perm[i] : i;
+        const float sg = (transpose && signs && signs[dst] < 0) ? -1.f : 1.f;
+        T *col = xt + dst;
+        for (int r = 0; r < rows; ++r) col[(int64_t)r * d] = from_f32<T>(sg * v[r * d + i]);
+    }
+}
+
+template <typename T, int NT, bool BIG>
+harp_status_t launch_blockowner(const harp_plan *plan, void *x, int64_t n_rows, int transpose, cudaStream_t stream) {
+    auto kern = harp_blockowner_kernel<T, NT, BIG>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+        return HARP_ERR_CUDA;
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int64_t d = plan->d;
+    int64_t r = (227 * 1024) / (d * (int64_t)sizeof(float));            // what shared memory holds
+    r = std::min<int64_t>(r, (n_rows + sms - 1) / sms);                 // one wave when the batch allows it
+    r = std::max<int64_t>(1, std::min<int64_t>(r, 64));
+    const int64_t grid = (n_rows + r - 1) / r;
+    if (grid > 0x7fffffffLL) return HARP_ERR_BAD_DIM;
+    kern<<<(unsigned)grid, NT, (size_t)r * d * sizeof(float), stream>>>((T *)x, n_rows, (int)d, (int)r, plan->st,
+                                                                              plan->d_blocks, plan->d_perm, plan->d_signs, transpose);
+    g_harp_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? HARP_OK : HARP_ERR_CUDA;
+}
+
 template <typename T, int ITEMS>
 harp_status_t launch(const harp_plan *plan, void *x, int64_t n_rows, int rows_per_cta, int transpose,
                      cudaStream_t stream) {
@@ -126,6 +231,16 @@ harp_status_t harp_generic_apply(const harp_plan *plan, void *x, int64_t n_rows,
     harp_status_t ok = harp_generic_supported(plan, dtype);
     if (ok != HARP_OK) return ok;
     const int64_t d = plan->d;
+    int max_radix = 0;
+    for (int t = 0; t < plan->st.m; ++t) max_radix = std::max(max_radix, (int)plan->st.b[t]);
+    if (max_radix <= 4) {      // 1024 threads, 64 registers: the block kernel takes at most 16 of them
+        return dtype == HARP_F32 ? launch_blockowner<float, 1024, false>(plan, x, n_rows, transpose, stream)
+                                 : launch_blockowner<__nv_bfloat16, 1024, false>(plan, x, n_rows, transpose, stream);
+    }
+    if (max_radix <= 8) {      // 256 threads so that an 8 x 8 block kernel stays in registers
+        return dtype == HARP_F32 ? launch_blockowner<float, 256, true>(plan, x, n_rows, transpose, stream)
+                                 : launch_blockowner<__nv_bfloat16, 256, true>(plan, x, n_rows, transpose, stream);
+    }
     // rows per CTA: as many as registers (kMaxItems) and shared memory allow, at most 8,
     // but keep at least ~2 CTAs per SM in flight when the batch is small.
     int r = (int)((int64_t)kThreads * kMaxItems / d);
