@@ -120,6 +120,7 @@ extern "C" harp_status_t harp_plan_create(harp_plan_t **out, int64_t d, int32_t 
     if (st == HARP_OK && p->d_signs &&
         cudaMemcpy(p->d_signs, p->h_signs.data(), (size_t)d, cudaMemcpyHostToDevice) != cudaSuccess)
         st = HARP_ERR_CUDA;
+    if (st == HARP_OK) st = harp_generic_build(p);
     if (st == HARP_OK) {
         harp_status_t fs = harp_fast_build(p);
         if (fs != HARP_OK && fs != HARP_ERR_UNSUPPORTED) st = fs;
@@ -148,6 +149,7 @@ extern "C" void harp_plan_destroy(harp_plan_t *p) {
             if (p->stage_buf[i]) cudaFree(p->stage_buf[i]);
         }
         if (p->d_blocks) cudaFree(p->d_blocks);
+        if (p->d_fused_blocks) cudaFree(p->d_fused_blocks);
         if (p->d_perm) cudaFree(p->d_perm);
         if (p->d_signs) cudaFree(p->d_signs);
     }

@@ -11,6 +11,7 @@
 #include <algorithm>
 
 #include "harp_internal.h"
+#include "harp_fuse.h"
 
 namespace {
 
@@ -155,6 +156,7 @@ harp_blockowner_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_ct
         const int src = (!transpose && perm) ? perm[i] : i;
         const float sg = (!transpose && signs && signs[src] < 0) ? -1.f : 1.f;
         const T *col = xt + src;
+#pragma unroll 4
         for (int r = 0; r < rows; ++r) v[r * d + i] = sg * to_f32<T>(col[(int64_t)r * d]);
     }
     __syncthreads();
@@ -178,12 +180,14 @@ harp_blockowner_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_ct
         const int dst = (transpose && perm) ? perm[i] : i;
         const float sg = (transpose && signs && signs[dst] < 0) ? -1.f : 1.f;
         T *col = xt + dst;
+#pragma unroll 4
         for (int r = 0; r < rows; ++r) col[(int64_t)r * d] = from_f32<T>(sg * v[r * d + i]);
     }
 }
 
 template <typename T, int NT, bool BIG>
-harp_status_t launch_blockowner(const harp_plan *plan, void *x, int64_t n_rows, int transpose, cudaStream_t stream) {
+harp_status_t launch_blockowner(const harp_plan *plan, const StageTable &st, const float *blocks, void *x, int64_t n_rows,
+                                int transpose, cudaStream_t stream) {
     auto kern = harp_blockowner_kernel<T, NT, BIG>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
         return HARP_ERR_CUDA;
@@ -191,13 +195,15 @@ harp_status_t launch_blockowner(const harp_plan *plan, void *x, int64_t n_rows, 
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const int64_t d = plan->d;
-    int64_t r = (227 * 1024) / (d * (int64_t)sizeof(float));            // what shared memory holds
-    r = std::min<int64_t>(r, (n_rows + sms - 1) / sms);                 // one wave when the batch allows it
+    const int per_sm = 1;                                               // CTAs per SM (see __launch_bounds__)
+    int64_t r = ((227 * 1024) / per_sm - 1024) / (d * (int64_t)sizeof(float));   // what shared memory holds
+    if (r < 1) r = (227 * 1024) / (d * (int64_t)sizeof(float));
+    r = std::min<int64_t>(r, (n_rows + (int64_t)sms * per_sm - 1) / ((int64_t)sms * per_sm));   // one wave when the batch allows it
     r = std::max<int64_t>(1, std::min<int64_t>(r, 64));
     const int64_t grid = (n_rows + r - 1) / r;
     if (grid > 0x7fffffffLL) return HARP_ERR_BAD_DIM;
-    kern<<<(unsigned)grid, NT, (size_t)r * d * sizeof(float), stream>>>((T *)x, n_rows, (int)d, (int)r, plan->st,
-                                                                              plan->d_blocks, plan->d_perm, plan->d_signs, transpose);
+    kern<<<(unsigned)grid, NT, (size_t)r * d * sizeof(float), stream>>>((T *)x, n_rows, (int)d, (int)r, st,
+                                                                              blocks, plan->d_perm, plan->d_signs, transpose);
     g_harp_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HARP_OK : HARP_ERR_CUDA;
 }
@@ -219,6 +225,54 @@ harp_status_t launch(const harp_plan *plan, void *x, int64_t n_rows, int rows_pe
 
 }  // namespace
 
+// Fuse runs of consecutive stages whose radices multiply to at most 4 into one dense stage (the
+// product of their block kernels on the coordinates they touch, computed in fp64, rounded once to
+// fp32): the same linear map with fewer stages, i.e. fewer barriers and shared-memory round trips.
+harp_status_t harp_generic_build(harp_plan *plan) {
+    const int m = plan->st.m;
+    const int64_t d = plan->d;
+    std::vector<harp_fuse::HostPhase> groups;
+    for (int t = 0; t < m;) {
+        int64_t prod = plan->st.b[t];
+        int t1 = t + 1;
+        while (t1 < m && prod * plan->st.b[t1] <= 4) prod *= plan->st.b[t1++];
+        groups.push_back({t, t1, (int)prod, plan->st.s[t], 0, 1});
+        t = t1;
+    }
+    if ((int)groups.size() == m) return HARP_OK;                       // nothing to fuse
+    StageTable ft{};
+    ft.m = (int32_t)groups.size();
+    int64_t off = 0;
+    for (size_t k = 0; k < groups.size(); ++k) {
+        ft.b[k] = groups[k].B;
+        ft.s[k] = (int32_t)groups[k].S;
+        ft.off[k] = off;
+        off += d * groups[k].B;
+    }
+    std::vector<float> fb;
+    try {
+        fb.resize((size_t)off);
+    } catch (const std::bad_alloc &) {
+        return HARP_ERR_ALLOC;
+    }
+    std::vector<double> F;
+    for (size_t k = 0; k < groups.size(); ++k) {
+        const int B = groups[k].B;
+        const int64_t S = groups[k].S;
+        for (int64_t c = 0; c < d / B; ++c) {
+            const int64_t alpha = c / S, beta = c % S;
+            harp_fuse::fused_block(plan, groups[k], alpha * B * S + beta, F);
+            float *dst = fb.data() + ft.off[k] + c * B * B;
+            for (int i = 0; i < B * B; ++i) dst[i] = (float)F[(size_t)i];
+        }
+    }
+    if (cudaMalloc(&plan->d_fused_blocks, sizeof(float) * (size_t)off) != cudaSuccess) return HARP_ERR_ALLOC;
+    if (cudaMemcpy(plan->d_fused_blocks, fb.data(), sizeof(float) * (size_t)off, cudaMemcpyHostToDevice) != cudaSuccess)
+        return HARP_ERR_CUDA;
+    plan->fused = ft;
+    return HARP_OK;
+}
+
 harp_status_t harp_generic_supported(const harp_plan *plan, harp_dtype_t dtype) {
     (void)dtype;
     if (plan->d > (int64_t)kThreads * kMaxItems) return HARP_ERR_UNSUPPORTED;
@@ -231,15 +285,18 @@ harp_status_t harp_generic_apply(const harp_plan *plan, void *x, int64_t n_rows,
     harp_status_t ok = harp_generic_supported(plan, dtype);
     if (ok != HARP_OK) return ok;
     const int64_t d = plan->d;
+    const bool use_fused = plan->fused.m > 0 && plan->d_fused_blocks;
+    const StageTable &bst = use_fused ? plan->fused : plan->st;
+    const float *bblk = use_fused ? plan->d_fused_blocks : plan->d_blocks;
     int max_radix = 0;
-    for (int t = 0; t < plan->st.m; ++t) max_radix = std::max(max_radix, (int)plan->st.b[t]);
+    for (int t = 0; t < bst.m; ++t) max_radix = std::max(max_radix, (int)bst.b[t]);
     if (max_radix <= 4) {      // 1024 threads, 64 registers: the block kernel takes at most 16 of them
-        return dtype == HARP_F32 ? launch_blockowner<float, 1024, false>(plan, x, n_rows, transpose, stream)
-                                 : launch_blockowner<__nv_bfloat16, 1024, false>(plan, x, n_rows, transpose, stream);
+        return dtype == HARP_F32 ? launch_blockowner<float, 1024, false>(plan, bst, bblk, x, n_rows, transpose, stream)
+                                 : launch_blockowner<__nv_bfloat16, 1024, false>(plan, bst, bblk, x, n_rows, transpose, stream);
     }
     if (max_radix <= 8) {      // 256 threads so that an 8 x 8 block kernel stays in registers
-        return dtype == HARP_F32 ? launch_blockowner<float, 256, true>(plan, x, n_rows, transpose, stream)
-                                 : launch_blockowner<__nv_bfloat16, 256, true>(plan, x, n_rows, transpose, stream);
+        return dtype == HARP_F32 ? launch_blockowner<float, 256, true>(plan, bst, bblk, x, n_rows, transpose, stream)
+                                 : launch_blockowner<__nv_bfloat16, 256, true>(plan, bst, bblk, x, n_rows, transpose, stream);
     }
     // rows per CTA: as many as registers (kMaxItems) and shared memory allow, at most 8,
     // but keep at least ~2 CTAs per SM in flight when the batch is small.

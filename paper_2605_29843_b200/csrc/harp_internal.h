@@ -29,6 +29,10 @@ struct harp_plan {
     StageTable st{};
     int64_t n_params = 0;
     float *d_blocks = nullptr;        // [sum_t d*b_t] fp32, stage after stage
+    // the same map with runs of small-radix stages fused into dense blocks of size <= 4 (fewer
+    // stages for the CUDA-core kernel); fused.m == 0 if nothing could be fused
+    StageTable fused{};
+    float *d_fused_blocks = nullptr;
     int32_t *d_perm = nullptr;        // nullptr = identity
     int8_t *d_signs = nullptr;        // nullptr = all +1
     // host copies (used to derive kernel-specific layouts)
@@ -46,6 +50,7 @@ struct harp_plan {
 extern std::atomic<int64_t> g_harp_launches;
 
 // generic CUDA-core path (harp_generic.cu)
+harp_status_t harp_generic_build(harp_plan *plan);   // fused stage table for the block-owner kernel
 harp_status_t harp_generic_supported(const harp_plan *plan, harp_dtype_t dtype);
 harp_status_t harp_generic_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype,
                                  int transpose, cudaStream_t stream);
