@@ -129,6 +129,10 @@ extern "C" harp_status_t harp_plan_create(harp_plan_t **out, int64_t d, int32_t 
         harp_status_t fs = harp_split_build(p);
         if (fs != HARP_OK && fs != HARP_ERR_UNSUPPORTED) st = fs;
     }
+    if (st == HARP_OK) {
+        harp_status_t fs = harp_col_build(p);
+        if (fs != HARP_OK && fs != HARP_ERR_UNSUPPORTED) st = fs;
+    }
     if (st != HARP_OK) {
         cudaGetLastError();
         harp_plan_destroy(p);
@@ -144,6 +148,7 @@ extern "C" void harp_plan_destroy(harp_plan_t *p) {
         DeviceGuard g(p->device);
         harp_fast_destroy(p);
         harp_split_destroy(p);
+        harp_col_destroy(p);
         for (int i = 0; i < 2; ++i) {
             if (p->stage_stream[i]) { cudaStreamSynchronize(p->stage_stream[i]); cudaStreamDestroy(p->stage_stream[i]); }
             if (p->stage_buf[i]) cudaFree(p->stage_buf[i]);
@@ -201,6 +206,13 @@ extern "C" harp_status_t harp_apply_two_sided(void *W, harp_dtype_t dtype, const
     if (scratch && (reinterpret_cast<uintptr_t>(scratch) & 255u) != 0) return HARP_ERR_BAD_DIM;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int64_t d_out = plan_out->d, d_in = plan_in->d;
+    // row side: every row of W through Q_in
+    harp_status_t st = harp_apply(plan_in, W, d_out, dtype, 0, s);
+    if (st != HARP_OK) return st;
+    // column side: every column of W through Q_out -- in place with the column kernels when the
+    // plan has them (no scratch needed), otherwise as rows of W^T (transpose, apply, transpose back)
+    st = harp_col_apply(plan_out, W, d_in, d_in, dtype, s);
+    if (st != HARP_ERR_UNSUPPORTED) return st;
     bool own = false;
     if (!scratch) {
         if (cudaMallocAsync(&scratch, (size_t)harp_two_sided_scratch_bytes(plan_out, plan_in, dtype), s) != cudaSuccess) {
@@ -209,10 +221,7 @@ extern "C" harp_status_t harp_apply_two_sided(void *W, harp_dtype_t dtype, const
         }
         own = true;
     }
-    // row side: every row of W through Q_in
-    harp_status_t st = harp_apply(plan_in, W, d_out, dtype, 0, s);
-    // column side: every column of W through Q_out (W^T rows, transposed back)
-    if (st == HARP_OK) st = harp_transpose_matrix(W, scratch, d_out, d_in, dtype, s);
+    st = harp_transpose_matrix(W, scratch, d_out, d_in, dtype, s);
     if (st == HARP_OK) st = harp_apply(plan_out, scratch, d_in, dtype, 0, s);
     if (st == HARP_OK) st = harp_transpose_matrix(scratch, W, d_in, d_out, dtype, s);
     if (own && cudaFreeAsync(scratch, s) != cudaSuccess && st == HARP_OK) st = HARP_ERR_CUDA;

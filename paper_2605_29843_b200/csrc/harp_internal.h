@@ -22,6 +22,7 @@ struct StageTable {
 
 struct FastPlan;   // tensor-core path data, whole rows per CTA (harp_fast.cu)
 struct SplitPlan;  // tensor-core path data, two passes over column groups (harp_split.cu)
+struct ColPlan;    // tensor-core path data for applying the plan down the columns of a matrix (harp_col.cu)
 
 struct harp_plan {
     int64_t d = 0;
@@ -41,6 +42,7 @@ struct harp_plan {
     std::vector<float> h_blocks;
     FastPlan *fast = nullptr;
     SplitPlan *split = nullptr;
+    ColPlan *col = nullptr;
     // staging owned by harp_apply_host
     void *stage_buf[2] = {nullptr, nullptr};
     int64_t stage_bytes = 0;
@@ -66,6 +68,13 @@ harp_status_t harp_split_build(harp_plan *plan);
 void harp_split_destroy(harp_plan *plan);
 harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype,
                                int transpose, cudaStream_t stream);
+
+// column-side apply for two-sided processing (harp_col.cu): plan applied down the columns of a
+// dim(plan) x n_cols row-major matrix with leading dimension ld
+harp_status_t harp_col_build(harp_plan *plan);
+void harp_col_destroy(harp_plan *plan);
+harp_status_t harp_col_apply(const harp_plan *plan, void *W, int64_t n_cols, int64_t ld, harp_dtype_t dtype,
+                             cudaStream_t stream);
 
 // out-of-place matrix transpose, rows x cols -> cols x rows (harp_two_sided.cu)
 harp_status_t harp_transpose_matrix(const void *src, void *dst, int64_t rows, int64_t cols,

@@ -99,3 +99,26 @@ def test_split_kernel_reports_unsupported(radices, perm):
     x = torch.zeros((16, spec.d), device="cuda", dtype=torch.bfloat16)
     st = harp.lib().harp_apply_ex(plan.handle, x.data_ptr(), 16, 1, 0, harp.KERNEL_SPLIT, None)
     assert st == harp.HARP_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("out_radices,in_radices", [((8, 8, 8, 8, 2), (4, 4, 4)), ((16, 16, 8, 7), (8, 9)),
+                                                    ((8, 8, 8, 8, 7), (8, 8)), ((4, 4, 4), (16, 16, 8)),
+                                                    ((16, 4, 3, 5), (8, 5)), ((8, 8, 8, 8), (8, 8, 8, 8))])
+def test_two_sided_with_column_kernels(out_radices, in_radices):
+    """plan_out without permutation and d_in a multiple of 8: the column side runs in place."""
+    from oracle import c_oracle
+    from harp_testlib import to_device, to_host_f64
+    p_out = wl.make_plan(51, int(np.prod(out_radices)), out_radices, "qr", perm="identity", signs=True)
+    p_in = wl.make_plan(52, int(np.prod(in_radices)), in_radices, "qr", perm="identity", signs=True)
+    rng = np.random.default_rng(12)
+    wh = host_rows(rng.standard_normal((p_out.d, p_in.d)), "bf16")
+    w64 = promote(wh, "bf16")
+    wd = to_device(wh, "bf16")
+    before = harp.harp_launch_count()
+    harp.two_sided_(wd, harp.plan_from_spec(p_out), harp.plan_from_spec(p_in))
+    torch.cuda.synchronize()
+    assert harp.harp_launch_count() - before <= 4          # no transposes: at most two passes per side
+    want = c_oracle.two_sided(c_oracle.CPlan(p_out), c_oracle.CPlan(p_in), w64)
+    got = to_host_f64(wd)
+    scale = np.minimum(np.linalg.norm(want, axis=1, keepdims=True), np.linalg.norm(want, axis=0, keepdims=True))
+    assert np.max(np.abs(got - want) / scale) <= 2 * TOL["bf16"]
