@@ -350,11 +350,21 @@ def run_profile_case(args):
     import paper_2605_29843_b200 as harp
     kernel = {"auto": harp.KERNEL_AUTO, "generic": harp.KERNEL_GENERIC, "fast": harp.KERNEL_FAST,
               "split": harp.KERNEL_SPLIT}[args.kernel]
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(7)
+    if args.profile_config == 6:          # two-sided processing of configuration 5's weight matrix
+        w = wl.config(5)
+        p_out, p_in = harp.plan_from_spec(w.plans["out"]), harp.plan_from_spec(w.plans["in"])
+        W = (torch.randn((p_out.d, p_in.d), generator=gen, device="cuda") * 0.02).to(torch.bfloat16)
+        for _ in range(args.profile_reps):
+            harp.two_sided_(W, p_out, p_in)
+        torch.cuda.synchronize()
+        print(json.dumps({"profile_case": "two_sided_8192x28672", "reps": args.profile_reps,
+                          "launches": harp.harp_launch_count()}))
+        return
     w = wl.config(args.profile_config)
     spec = w.plans["in"] if args.profile_config == 5 else w.plans["q"]
     plan = harp.plan_from_spec(spec)
-    gen = torch.Generator(device="cuda")
-    gen.manual_seed(7)
     tdt = torch.float32 if w.data["x"].dtype == "f32" else torch.bfloat16
     x = torch.randn((args.profile_rows, spec.d), generator=gen, device="cuda").to(tdt)
     for i in range(args.profile_reps):

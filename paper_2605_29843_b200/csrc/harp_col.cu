@@ -72,7 +72,7 @@ harp_col_kernel(__nv_bfloat16 *__restrict__ W, int64_t ld, int64_t n_cols, ColPa
     extern __shared__ __align__(16) unsigned char smem_raw[];
     const uint32_t sbase = smem_u32(smem_raw);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int rowbytes = P.rowbytes, NC = P.NC, MT = NC >> 4, mt_shift = NC == 64 ? 2 : 1;
+    const int rowbytes = P.rowbytes, NC = P.NC, MT = NC >> 4;
     const size_t tile_bytes = (size_t)P.n_rows_phys * rowbytes;          // includes one scratch row for padded slots
     int32_t *tab_s = reinterpret_cast<int32_t *>(smem_raw + tile_bytes);
     const uint32_t bf_s = sbase + (uint32_t)((tile_bytes + (size_t)P.tables_len * 4 + 15) / 16 * 16);
@@ -105,42 +105,45 @@ harp_col_kernel(__nv_bfloat16 *__restrict__ W, int64_t ld, int64_t n_cols, ColPa
 
         for (int p = 0; p < P.n_phases; ++p) {
             const ColPhase &ph = P.ph[p];
-            const int n_work = ph.n_items * MT;
+            // a warp takes a block through all 16-column groups of the tile: the block's fragment and
+            // addresses are set up once
             if (ph.B == 16) {
                 const int k = (lane & 7) + 8 * (lane >> 4), mch = (lane >> 3) & 1;
                 const bool real = k < ph.B_real;
-                const uint32_t lane_ld = (uint32_t)((real ? k * ph.wr : 0) * rowbytes + 16 * mch);
-                for (int w = warp; w < n_work; w += kColWarps) {
-                    const int it = w >> mt_shift, mt = w & (MT - 1);
-                    const int base_row = tab_s[ph.items_off + it];
-                    const uint32_t tile_off = sbase + (uint32_t)(32 * mt);
+                const uint32_t lane_ld = sbase + (uint32_t)((real ? k * ph.wr : 0) * rowbytes + 16 * mch);
+                const uint32_t lane_scr = sbase + (uint32_t)(scratch_row * rowbytes + 16 * mch);
+                for (int it = warp; it < ph.n_items; it += kColWarps) {
+                    const uint32_t row_off = (uint32_t)(tab_s[ph.items_off + it] * rowbytes);
                     const uint4 bf = lds128(bf_s + 4u * (uint32_t)(ph.bfrag_off + (it * 32 + lane) * 4));
-                    uint32_t a[4];
-                    ldmatrix_x4_t(a, tile_off + (uint32_t)(base_row * rowbytes) + lane_ld);
-                    float c0f[4], c1f[4];
-                    mma_k16(c0f, a, bf.x, bf.y);
-                    mma_k16(c1f, a, bf.z, bf.w);
-                    const uint32_t st_addr = real ? tile_off + (uint32_t)(base_row * rowbytes) + lane_ld
-                                                  : tile_off + (uint32_t)(scratch_row * rowbytes + 16 * mch);
-                    stmatrix_x4_t(st_addr, pack_bf16(c0f[0], c0f[1]), pack_bf16(c0f[2], c0f[3]), pack_bf16(c1f[0], c1f[1]),
-                                  pack_bf16(c1f[2], c1f[3]));
+                    uint32_t ld_addr = lane_ld + row_off, st_addr = real ? ld_addr : lane_scr;
+#pragma unroll 2
+                    for (int mt = 0; mt < MT; ++mt, ld_addr += 32, st_addr += 32) {
+                        uint32_t a[4];
+                        ldmatrix_x4_t(a, ld_addr);
+                        float c0f[4], c1f[4];
+                        mma_k16(c0f, a, bf.x, bf.y);
+                        mma_k16(c1f, a, bf.z, bf.w);
+                        stmatrix_x4_t(st_addr, pack_bf16(c0f[0], c0f[1]), pack_bf16(c0f[2], c0f[3]), pack_bf16(c1f[0], c1f[1]),
+                                      pack_bf16(c1f[2], c1f[3]));
+                    }
                 }
             } else {
                 const int k = lane & 7, mch = (lane >> 3) & 1;
                 const bool real = k < ph.B_real;
-                const uint32_t lane_ld = (uint32_t)((real ? k * ph.wr : 0) * rowbytes + 16 * mch);
-                for (int w = warp; w < n_work; w += kColWarps) {
-                    const int it = w >> mt_shift, mt = w & (MT - 1);
-                    const int base_row = tab_s[ph.items_off + it];
-                    const uint32_t tile_off = sbase + (uint32_t)(32 * mt);
+                const uint32_t lane_ld = sbase + (uint32_t)((real ? k * ph.wr : 0) * rowbytes + 16 * mch);
+                const uint32_t lane_scr = sbase + (uint32_t)(scratch_row * rowbytes + 16 * mch);
+                for (int it = warp; it < ph.n_items; it += kColWarps) {
+                    const uint32_t row_off = (uint32_t)(tab_s[ph.items_off + it] * rowbytes);
                     const uint32_t bf = lds32c(bf_s + 4u * (uint32_t)(ph.bfrag_off + it * 32 + lane));
-                    uint32_t a[2];
-                    ldmatrix_x2_t(a, tile_off + (uint32_t)(base_row * rowbytes) + lane_ld);
-                    float c0f[4];
-                    mma_k8(c0f, a, bf);
-                    const uint32_t st_addr = real ? tile_off + (uint32_t)(base_row * rowbytes) + lane_ld
-                                                  : tile_off + (uint32_t)(scratch_row * rowbytes + 16 * mch);
-                    stmatrix_x2_t(st_addr, pack_bf16(c0f[0], c0f[1]), pack_bf16(c0f[2], c0f[3]));
+                    uint32_t ld_addr = lane_ld + row_off, st_addr = real ? ld_addr : lane_scr;
+#pragma unroll 2
+                    for (int mt = 0; mt < MT; ++mt, ld_addr += 32, st_addr += 32) {
+                        uint32_t a[2];
+                        ldmatrix_x2_t(a, ld_addr);
+                        float c0f[4];
+                        mma_k8(c0f, a, bf);
+                        stmatrix_x2_t(st_addr, pack_bf16(c0f[0], c0f[1]), pack_bf16(c0f[2], c0f[3]));
+                    }
                 }
             }
             __syncthreads();
