@@ -74,6 +74,54 @@ harp_status_t harp_plan_create(harp_plan_t **out, int64_t d, int32_t n_stages,
                                const int32_t *radices, const int32_t *perm,
                                const int8_t *signs, const float *const *blocks);
 
+/* Greedy Mixed-Radix schedule (Algorithm 2, appendix "Stage schedules and Mixed-Radix
+ * construction"): peel the preferred radix b_base while it divides d, then the largest factors
+ * <= b_max down to 2, then the leftover factor as one last stage.
+ *   radices  HOST int32[max_stages], receives the schedule
+ * Returns the number of stages, or -1 (d < 2, a radix bound < 2, NULL, or max_stages too small). */
+int32_t harp_greedy_schedule(int64_t d, int32_t b_base, int32_t b_max, int32_t *radices,
+                             int32_t max_stages);
+
+/* Parameters per block of radix b: 1 (Givens angle) for b = 2, b(b-1)/2 (strict upper triangle of
+ * the skew-symmetric matrix A, row-major, i < j) otherwise (Eq. 10, 11, 13). */
+int32_t harp_theta_params_per_block(int32_t b);
+
+/* Block kernels of one stage from stored parameters, B_c = Q(theta_c) G_b (Eq. 9): Q is the Givens
+ * rotation [[cos,-sin],[sin,cos]] for b = 2 (Eq. 10) and the Cayley map (I+A)^{-1}(I-A) for b > 2
+ * (Eq. 11).  All pointers HOST; no CUDA call is made.
+ *   theta     float[n_blocks][n_par] or NULL
+ *   theta_q   int8[n_blocks][n_par] with scales float[n_blocks] (int8 storage of the appendix:
+ *             a = scale * q), used when theta is NULL
+ *   mixer     float[b][b] orthogonal base mixer G_b, or NULL for the normalised Sylvester Hadamard
+ *             matrix (b a power of two; otherwise HARP_ERR_NULL)
+ *   out_blocks float[n_blocks][b][b], the layout harp_plan_create expects
+ * Arithmetic in fp64, one rounding to fp32. */
+harp_status_t harp_blocks_from_theta(int32_t b, int64_t n_blocks, const float *theta,
+                                     const int8_t *theta_q, const float *scales,
+                                     const float *mixer, float *out_blocks);
+
+/* harp_plan_create with every stage's blocks rebuilt by harp_blocks_from_theta.  theta, theta_q,
+ * scales, mixers are HOST arrays of n_stages pointers (theta or theta_q may be NULL as a whole;
+ * mixers may be NULL if every radix is a power of two). */
+harp_status_t harp_plan_create_from_theta(harp_plan_t **out, int64_t d, int32_t n_stages,
+                                          const int32_t *radices, const int32_t *perm,
+                                          const int8_t *signs, const float *const *theta,
+                                          const int8_t *const *theta_q,
+                                          const float *const *scales,
+                                          const float *const *mixers);
+
+/* Kronecker fallback (Eq. 12): the plan of dimension d = K * n2 equal to
+ * (H~_K / sqrt K) (x) T_{n2}: the stages of the n2-plan act on each of the K contiguous runs of n2
+ * coordinates, then one radix-K stage of stride n2 mixes the runs with the fixed table.
+ *   radices, blocks_n2  HOST description of T_{n2} as for harp_plan_create
+ *   hk       HOST float[K][K] with entries +1/-1 and H H^T = K I (else HARP_ERR_BAD_SIGNS /
+ *            HARP_ERR_BAD_SCHEDULE); used as out[k'] = sum_k in[k] H[k][k'] / sqrt K
+ *   perm, signs  over d, as for harp_plan_create */
+harp_status_t harp_plan_create_kronecker(harp_plan_t **out, int64_t n2, int32_t n_stages,
+                                         const int32_t *radices, const float *const *blocks_n2,
+                                         int32_t K, const float *hk, const int32_t *perm,
+                                         const int8_t *signs);
+
 /* Release the plan and its device memory.  NULL is allowed. */
 void harp_plan_destroy(harp_plan_t *plan);
 

@@ -39,6 +39,16 @@ def lib() -> ctypes.CDLL:
         vp, i64, i32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32
         L.harp_plan_create.restype = ctypes.c_int
         L.harp_plan_create.argtypes = [ctypes.POINTER(vp), i64, i32, vp, vp, vp, ctypes.POINTER(vp)]
+        L.harp_greedy_schedule.restype = i32
+        L.harp_greedy_schedule.argtypes = [i64, i32, i32, vp, i32]
+        L.harp_theta_params_per_block.restype = i32
+        L.harp_theta_params_per_block.argtypes = [i32]
+        L.harp_blocks_from_theta.restype = ctypes.c_int
+        L.harp_blocks_from_theta.argtypes = [i32, i64, vp, vp, vp, vp, vp]
+        L.harp_plan_create_from_theta.restype = ctypes.c_int
+        L.harp_plan_create_from_theta.argtypes = [ctypes.POINTER(vp), i64, i32, vp, vp, vp, vp, vp, vp, vp]
+        L.harp_plan_create_kronecker.restype = ctypes.c_int
+        L.harp_plan_create_kronecker.argtypes = [ctypes.POINTER(vp), i64, i32, vp, ctypes.POINTER(vp), i32, vp, vp, vp]
         L.harp_plan_destroy.restype = None
         L.harp_plan_destroy.argtypes = [vp]
         L.harp_plan_dim.restype = i64
@@ -111,6 +121,75 @@ def harp_plan_create(d: int, radices: Sequence[int], perm=None, signs=None, bloc
     if st != HARP_OK:
         raise HarpError(st, "harp_plan_create")
     return plan
+
+
+def harp_greedy_schedule(d: int, b_base: int = 8, b_max: int = 8):
+    buf = (ctypes.c_int32 * 64)()
+    n = lib().harp_greedy_schedule(int(d), int(b_base), int(b_max), buf, 64)
+    if n < 0:
+        raise HarpError(3, "harp_greedy_schedule")
+    return [int(buf[i]) for i in range(n)]
+
+
+def harp_theta_params_per_block(b: int) -> int:
+    return int(lib().harp_theta_params_per_block(int(b)))
+
+
+def _ptr_array(arrs):
+    if arrs is None:
+        return None, None
+    keep = [None if a is None else np.ascontiguousarray(a) for a in arrs]
+    return (ctypes.c_void_p * len(keep))(*[None if a is None else a.ctypes.data for a in keep]), keep
+
+
+def harp_blocks_from_theta(b: int, theta=None, theta_q=None, scales=None, mixer=None) -> np.ndarray:
+    """Host-only: blocks[n_blocks, b, b] (float32) from per-block parameters."""
+    npar = harp_theta_params_per_block(b)
+    th = None if theta is None else np.ascontiguousarray(theta, dtype=np.float32).reshape(-1, npar)
+    tq = None if theta_q is None else np.ascontiguousarray(theta_q, dtype=np.int8).reshape(-1, npar)
+    sc = None if scales is None else np.ascontiguousarray(scales, dtype=np.float32)
+    mx = None if mixer is None else np.ascontiguousarray(mixer, dtype=np.float32)
+    n = (th if th is not None else tq).shape[0]
+    out = np.empty((n, b, b), dtype=np.float32)
+    st = lib().harp_blocks_from_theta(int(b), n, None if th is None else th.ctypes.data,
+                                      None if tq is None else tq.ctypes.data, None if sc is None else sc.ctypes.data,
+                                      None if mx is None else mx.ctypes.data, out.ctypes.data)
+    if st != HARP_OK:
+        raise HarpError(st, "harp_blocks_from_theta")
+    return out
+
+
+def harp_plan_create_from_theta(d: int, radices: Sequence[int], perm=None, signs=None, theta=None, theta_q=None,
+                                scales=None, mixers=None) -> Plan:
+    rad = np.ascontiguousarray(radices, dtype=np.int32)
+    pm = None if perm is None else np.ascontiguousarray(perm, dtype=np.int32)
+    sg = None if signs is None else np.ascontiguousarray(signs, dtype=np.int8)
+    th, k1 = _ptr_array(None if theta is None else [np.asarray(a, dtype=np.float32) for a in theta])
+    tq, k2 = _ptr_array(None if theta_q is None else [np.asarray(a, dtype=np.int8) for a in theta_q])
+    sc, k3 = _ptr_array(None if scales is None else [np.asarray(a, dtype=np.float32) for a in scales])
+    mx, k4 = _ptr_array(None if mixers is None else [None if a is None else np.asarray(a, dtype=np.float32) for a in mixers])
+    out = ctypes.c_void_p()
+    st = lib().harp_plan_create_from_theta(ctypes.byref(out), int(d), len(rad), rad.ctypes.data,
+                                           None if pm is None else pm.ctypes.data, None if sg is None else sg.ctypes.data,
+                                           th, tq, sc, mx)
+    if st != HARP_OK:
+        raise HarpError(st, "harp_plan_create_from_theta")
+    return Plan(out.value, int(d))
+
+
+def harp_plan_create_kronecker(n2: int, radices: Sequence[int], blocks_n2, K: int, hk, perm=None, signs=None) -> Plan:
+    rad = np.ascontiguousarray(radices, dtype=np.int32)
+    blks = [np.ascontiguousarray(b, dtype=np.float32) for b in blocks_n2]
+    arr = (ctypes.c_void_p * len(blks))(*[b.ctypes.data for b in blks])
+    h = np.ascontiguousarray(hk, dtype=np.float32)
+    pm = None if perm is None else np.ascontiguousarray(perm, dtype=np.int32)
+    sg = None if signs is None else np.ascontiguousarray(signs, dtype=np.int8)
+    out = ctypes.c_void_p()
+    st = lib().harp_plan_create_kronecker(ctypes.byref(out), int(n2), len(rad), rad.ctypes.data, arr, int(K), h.ctypes.data,
+                                          None if pm is None else pm.ctypes.data, None if sg is None else sg.ctypes.data)
+    if st != HARP_OK:
+        raise HarpError(st, "harp_plan_create_kronecker")
+    return Plan(out.value, int(K) * int(n2))
 
 
 def plan_from_spec(spec) -> Plan:

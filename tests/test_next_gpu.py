@@ -1,0 +1,88 @@
+"""Plan helpers and the symmetric two-sided product on the GPU, against the oracles."""
+import numpy as np
+import pytest
+import scipy.linalg
+import torch
+
+import paper_2605_29843_b200 as harp
+from oracle import harp_oracle as orc
+from oracle import harp_params as prm
+from paper_2605_29843_b200 import workloads as wl
+from harp_testlib import TOL, gpu_apply, host_rows, promote, to_device, to_host_f64
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("radices", [(2, 2, 2, 4), (8, 8), (4, 2, 8, 5), (16, 2)])
+@pytest.mark.parametrize("int8", [False, True])
+def test_plan_from_theta(radices, int8):
+    d = int(np.prod(radices))
+    rng = np.random.default_rng(17)
+    theta, mixers, blocks64, tq, sc = [], [], [], [], []
+    for b in radices:
+        th = rng.normal(0, 0.25, (d // b, prm.n_params(b)))
+        mixer = None if (b & (b - 1)) == 0 else np.linalg.qr(rng.standard_normal((b, b)))[0]
+        if int8:
+            q, s = prm.quantize_theta(th)
+            s = s.astype(np.float32)
+            tq.append(q); sc.append(s)
+            th = prm.dequantize_theta(q, s.astype(np.float64))
+        theta.append(th.astype(np.float32))
+        mixers.append(None if mixer is None else mixer.astype(np.float32))
+        blocks64.append(prm.blocks_from_theta(b, theta[-1].astype(np.float64) if not int8 else th,
+                                              None if mixer is None else mixer.astype(np.float32).astype(np.float64)))
+    signs = wl.rademacher(rng, d)
+    perm = rng.permutation(d).astype(np.int32)
+    plan = harp.harp_plan_create_from_theta(d, radices, perm, signs, theta=None if int8 else theta,
+                                            theta_q=tq if int8 else None, scales=sc if int8 else None, mixers=mixers)
+    oplan = orc.OraclePlan(d, radices, perm, signs, blocks64)
+    xh = host_rows(rng.standard_normal((13, d)), "f32")
+    got, guards = gpu_apply(plan, xh, "f32")
+    assert guards and orc.rel_err_rows(got, orc.forward(oplan, promote(xh, "f32"))) <= TOL["f32"]
+    got, guards = gpu_apply(plan, xh, "f32", True)
+    assert guards and orc.rel_err_rows(got, orc.transpose(oplan, promote(xh, "f32"))) <= TOL["f32"]
+
+
+@pytest.mark.parametrize("K,rows", [(2, None), (4, [1, 3, 0, 2]), (8, [5, 0, 7, 2, 1, 6, 3, 4])])
+def test_kronecker_fallback_plan(K, rows):
+    hk = scipy.linalg.hadamard(K).astype(np.float64)
+    if rows is not None:
+        hk = hk[rows]
+    radices, n2 = (4, 2, 4), 32
+    rng = np.random.default_rng(23)
+    blocks = [wl.qr_orthogonal(rng, n2 // b, b).astype(np.float32) for b in radices]
+    plan = harp.harp_plan_create_kronecker(n2, radices, blocks, K, hk)
+    d = K * n2
+    assert harp.harp_plan_dim(plan) == d
+    t_small = orc.dense(orc.OraclePlan(n2, radices, None, None, blocks))
+    want = np.kron(hk / np.sqrt(K), t_small)
+    eye = np.eye(d, dtype=np.float32)
+    got, guards = gpu_apply(plan, eye, "f32")                 # rows of I through the plan = the dense matrix
+    assert guards and np.max(np.abs(got - want)) < 2e-6
+    # a table that is not a Hadamard table is rejected
+    bad = hk.copy()
+    bad[0, 0] = -bad[0, 0]
+    with pytest.raises(harp.HarpError):
+        harp.harp_plan_create_kronecker(n2, radices, blocks, K, bad)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_symmetric_two_sided_product(dtype):
+    """H~ = V^T H V (second moment rotated on both sides with the same processor)."""
+    spec = wl.make_plan(61, 512, (8, 8, 8), "qr", perm="identity", signs=True)
+    V = orc.dense(orc.OraclePlan.from_spec(spec))
+    rng = np.random.default_rng(29)
+    X = rng.standard_normal((700, 512)) * (1.0 + 5.0 * (rng.random(512) < 0.02))
+    H = X.T @ X / 700.0
+    hh = host_rows(H, dtype)
+    h64 = promote(hh, dtype)
+    hd = to_device(hh, dtype)
+    plan = harp.plan_from_spec(spec)
+    harp.two_sided_(hd, plan, plan)
+    torch.cuda.synchronize()
+    got = to_host_f64(hd)
+    want = V.T @ h64 @ V
+    scale = np.minimum(np.linalg.norm(want, axis=1, keepdims=True), np.linalg.norm(want, axis=0, keepdims=True))
+    assert np.max(np.abs(got - want) / scale) <= 2 * TOL[dtype]
+    assert abs(np.trace(got) - np.trace(h64)) / np.trace(h64) < (1e-5 if dtype == "f32" else 5e-3)
+    assert np.max(np.abs(got - got.T) / scale) <= 4 * TOL[dtype]
