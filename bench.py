@@ -318,8 +318,9 @@ def run_gpu(args):
             "metric": METRIC, "value": world * 2 * n_rows * args.steps / dt_max, "unit": UNIT,
             "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
             "ms_per_step": 1e3 * dt_max / args.steps, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16 I/O, fp32 accumulate", "data": "synthetic",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "n_rows": n_rows, "d": d, "kernel": args.kernel,
+                       "arithmetic": "bf16 operands, fp32 accumulate, one rounding to bf16 per phase",
                        "l2": f"{N_BUF} rotating 134 MB buffers (inputs larger than L2)", "parallelism": f"rows x{world}"},
             "clocks": clocks,
             "e2e": {"value": world * 2 * n_rows * e2e_steps / e2e_dt, "unit": UNIT,
