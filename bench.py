@@ -214,6 +214,19 @@ def bench_extra_configs(torch, harp, kernel, peak):
                 torch.cuda.synchronize()
                 dt = time_region(torch, lambda i: harp.apply_(plan, x, kernel=kernel), 200)
                 dec[str(n)] = {"us_per_call": 1e6 * dt / 200}
+                # the same 100 calls replayed from one CUDA graph (no per-call launch cost on the host)
+                side = torch.cuda.Stream()
+                side.wait_stream(torch.cuda.current_stream())
+                with torch.cuda.stream(side):
+                    graph = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(graph, stream=side):
+                        for _ in range(100):
+                            harp.apply_(plan, x, kernel=kernel)
+                torch.cuda.current_stream().wait_stream(side)
+                graph.replay()
+                torch.cuda.synchronize()
+                dtg = time_region(torch, lambda i: graph.replay(), 5)
+                dec[str(n)]["us_per_call_cuda_graph"] = 1e6 * dtg / 500
             res["decode"] = dec
         if cfg == 5:
             del bufs
