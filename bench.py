@@ -242,6 +242,16 @@ def bench_extra_configs(torch, harp, kernel, peak):
             wbytes = 2 * wd.n_rows * wd.d * 2
             res["two_sided"] = {"ms": 1e3 * dt / 10, "GBps_vs_1R1W": wbytes * 10 / dt / 1e9,
                                 "frac_of_measured_peak_vs_1R1W": wbytes * 10 / dt / 1e9 / peak}
+            # diagnostics of the processed weight (Eq. 4): one read of W per call
+            acc = torch.zeros(4, dtype=torch.float64, device="cuda")
+            stream = torch.cuda.current_stream().cuda_stream
+            mu = lambda i: harp.harp_weight_incoherence(W.data_ptr(), wd.n_rows, wd.d, harp.HARP_BF16, acc.data_ptr(), stream)
+            for i in range(2):
+                mu(i)
+            dt = time_region(torch, mu, 10)
+            res["weight_incoherence"] = {"ms": 1e3 * dt / 10, "GBps_read": wbytes / 2 * 10 / dt / 1e9,
+                                         "frac_of_measured_peak": wbytes / 2 * 10 / dt / 1e9 / peak,
+                                         "mu_W": float(acc[0].item())}
         out[w.name] = res
         bufs = None
         torch.cuda.empty_cache()

@@ -182,6 +182,38 @@ harp_status_t harp_apply_two_sided_static(void *W, harp_dtype_t dtype,
 /* Capacity in bytes of the fixed scratch array used by harp_apply_two_sided_static. */
 int64_t harp_two_sided_static_capacity_bytes(void);
 
+/* ---- Diagnostics of a processed layer (appendix "Incoherence diagnostics") ----------------
+ * One pass over a row-major DEVICE matrix each; asynchronous on stream; nothing is allocated.
+ * out is a DEVICE array of four doubles, 8-byte aligned, owned by the caller: out[0] receives
+ * the result, out[1..3] the accumulators named below (the call zeroes all four first).
+ * Matrices are contiguous (leading dimension = number of columns) and aligned to their
+ * element size; 16-byte alignment with a column count that is a multiple of 16 bytes takes
+ * the vectorised path.  Errors: HARP_ERR_NULL, HARP_ERR_BAD_DIM (non-positive or > 2^31
+ * extents, misaligned pointers, block outside [1, n]), HARP_ERR_BAD_DTYPE, HARP_ERR_CUDA. */
+
+/* Weight incoherence, Eq. 4: mu_W(A) = sqrt(m n) * max|A_ij| / ||A||_F for A (m x n).
+ * out[1] = max|A_ij|, out[2] = ||A||_F^2; mu_W = 0 for the zero matrix. */
+harp_status_t harp_weight_incoherence(const void *A, int64_t m, int64_t n, harp_dtype_t dtype,
+                                      double *out, void *stream);
+
+/* Off-block energy of the rotated curvature proxy, Eq. 15:
+ * R_bd = (1/n^2) * sum over block pairs p != q of ||H_pq||_F^2, the blocks being the
+ * quantizer's contiguous partition of the n coordinates into runs of `block` (the last run
+ * may be shorter).  H is n x n (for instance the result of harp_apply_two_sided(H, V, V)).
+ * out[2] = ||H||_F^2, out[3] = sum of squared entries inside the diagonal blocks. */
+harp_status_t harp_offblock_energy(const void *H, int64_t n, int64_t block, harp_dtype_t dtype,
+                                   double *out, void *stream);
+
+/* Diagonal Hessian-weighted reconstruction proxy, Eq. 14:
+ * L_diag = 1/(d_out d_in) * sum_ij (Wt_ij - Wq_ij)^2 * wbar_j,  w_j = |H_jj|, wbar = w / mean(w).
+ *   Wt, Wq  DEVICE d_out x d_in, the rotated weight and its quantised copy (the quantizer is
+ *           the caller's; the paper treats Q(Wt) as a constant of the step)
+ *   H       DEVICE d_in x d_in of h_dtype, only its diagonal is read
+ * out[1] = sum_ij (Wt_ij - Wq_ij)^2 w_j, out[2] = sum_j w_j; L_diag = 0 if every w_j is 0. */
+harp_status_t harp_diag_weighted_error(const void *Wt, const void *Wq, int64_t d_out, int64_t d_in,
+                                       harp_dtype_t dtype, const void *H, harp_dtype_t h_dtype,
+                                       double *out, void *stream);
+
 /* Apply to rows that live in HOST memory (pinned memory gives full copy speed):
  * copies chunks host->device, applies, copies back, on two internal streams so that
  * copies overlap kernels; returns after the last copy has completed.  The device staging

@@ -65,6 +65,12 @@ def lib() -> ctypes.CDLL:
         L.harp_apply_two_sided_static.argtypes = [vp, ctypes.c_int, vp, vp, vp]
         L.harp_two_sided_static_capacity_bytes.restype = i64
         L.harp_two_sided_static_capacity_bytes.argtypes = []
+        L.harp_weight_incoherence.restype = ctypes.c_int
+        L.harp_weight_incoherence.argtypes = [vp, i64, i64, ctypes.c_int, vp, vp]
+        L.harp_offblock_energy.restype = ctypes.c_int
+        L.harp_offblock_energy.argtypes = [vp, i64, i64, ctypes.c_int, vp, vp]
+        L.harp_diag_weighted_error.restype = ctypes.c_int
+        L.harp_diag_weighted_error.argtypes = [vp, vp, i64, i64, ctypes.c_int, vp, ctypes.c_int, vp, vp]
         L.harp_apply_host.restype = ctypes.c_int
         L.harp_apply_host.argtypes = [vp, vp, i64, ctypes.c_int, ctypes.c_int]
         L.harp_launch_count.restype = i64
@@ -234,6 +240,29 @@ def harp_two_sided_static_capacity_bytes() -> int:
 
 def harp_two_sided_scratch_bytes(plan_out: Plan, plan_in: Plan, dtype: int) -> int:
     return int(lib().harp_two_sided_scratch_bytes(plan_out.handle, plan_in.handle, int(dtype)))
+
+
+def harp_weight_incoherence(a_ptr: int, m: int, n: int, dtype: int, out_ptr: int, stream: int = 0) -> None:
+    """Eq. 4 on a DEVICE m x n matrix; out_ptr: DEVICE double[4] (result in [0])."""
+    st = lib().harp_weight_incoherence(a_ptr, int(m), int(n), int(dtype), out_ptr, stream or None)
+    if st != HARP_OK:
+        raise HarpError(st, "harp_weight_incoherence")
+
+
+def harp_offblock_energy(h_ptr: int, n: int, block: int, dtype: int, out_ptr: int, stream: int = 0) -> None:
+    """Eq. 15 on a DEVICE n x n matrix with contiguous blocks of `block`; out_ptr: DEVICE double[4]."""
+    st = lib().harp_offblock_energy(h_ptr, int(n), int(block), int(dtype), out_ptr, stream or None)
+    if st != HARP_OK:
+        raise HarpError(st, "harp_offblock_energy")
+
+
+def harp_diag_weighted_error(wt_ptr: int, wq_ptr: int, d_out: int, d_in: int, dtype: int, h_ptr: int, h_dtype: int,
+                             out_ptr: int, stream: int = 0) -> None:
+    """Eq. 14 for DEVICE Wt, Wq (d_out x d_in) and H (d_in x d_in, diagonal only); out_ptr: DEVICE double[4]."""
+    st = lib().harp_diag_weighted_error(wt_ptr, wq_ptr, int(d_out), int(d_in), int(dtype), h_ptr, int(h_dtype),
+                                        out_ptr, stream or None)
+    if st != HARP_OK:
+        raise HarpError(st, "harp_diag_weighted_error")
 
 
 def harp_apply_host(plan: Plan, host_ptr: int, n_rows: int, dtype: int, transpose: bool = False) -> None:
