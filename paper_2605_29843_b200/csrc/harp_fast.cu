@@ -20,14 +20,20 @@
 // Mixed-radix digit reversal of the plan's own schedule: the tile is copied in coalesced in
 // source order, the phases run in place on the source-ordered layout (a digit reversal
 // maps every phase onto a digit group again, only with other strides), and the one phase
-// next to the output does the reordering inside shared memory: all of its operands are
-// read into registers, the CTA synchronises, and the results are written in output order.
+// next to the output does the reordering inside shared memory.  Forward: an item of that
+// phase reads eight blocks that are neighbours in output order (16 contiguous source values
+// each, ldmatrix) and writes its sixteen eight-block runs into the same sixteen 16-byte
+// slots, so the phase is in place and the copy to global memory follows a chunk map.
+// Transpose: all operands of the phase are read from an output-ordered layout into registers,
+// the CTA synchronises, and the results are written as contiguous source blocks (the in-place
+// form of this direction exists too, but measures slower).
 // Any other permutation that maps every aligned run of eight source coordinates onto the
 // same slot of eight different first-phase blocks is gathered (forward) or scattered
 // (transpose) in global memory with 16-byte accesses by the first/last phase.  All other
 // permutations use the generic kernel.
 #include <algorithm>
 #include <cmath>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <map>
@@ -48,8 +54,9 @@ enum PhaseMode : int32_t {
     MODE_SS = 1,   // strided block in shared memory, eight blocks per item, in place
     MODE_GS = 2,   // operands gathered from global memory, result to contiguous smem blocks
     MODE_CG = 3,   // operands from contiguous smem blocks, result scattered to global memory
-    MODE_PO = 4,   // contiguous smem blocks in, CTA barrier, strided smem out (reorders the tile)
-    MODE_PI = 5    // strided smem in, CTA barrier, contiguous smem blocks out (reorders the tile)
+    MODE_PO = 4,   // contiguous smem blocks in, eight-block runs out to the same slots (reorders the tile in place)
+    MODE_PI = 5,   // strided smem in (output-ordered layout), CTA barrier, contiguous smem blocks out
+    MODE_PI2 = 6   // eight-block runs in, contiguous smem blocks out to the same slots (in place)
 };
 
 struct PhaseDesc {
@@ -128,7 +135,16 @@ __device__ __forceinline__ void gs_store(const TileCtx &c, const PhaseDesc &ph, 
         stmatrix_x4(c.sbase + 2u * (uint32_t)(mrow * c.pitch + tab[e] + mcol), mats[e][0], mats[e][1], mats[e][2], mats[e][3]);
 }
 
-template <int NT>
+// MODES: bit m set = the code of phase mode m is compiled in.  The host launches the variant
+// that holds exactly the modes of the plan's direction, so that the register allocation of one
+// scheme does not pay for the others.
+__host__ __device__ constexpr uint32_t bit(int mode) { return 1u << mode; }
+constexpr uint32_t kModesGeneral = bit(MODE_CC) | bit(MODE_SS) | bit(MODE_GS) | bit(MODE_CG);
+constexpr uint32_t kModesReorderOut = bit(MODE_SS) | bit(MODE_PO);
+constexpr uint32_t kModesReorderIn = bit(MODE_SS) | bit(MODE_PI);
+constexpr uint32_t kModesReorderIn2 = bit(MODE_SS) | bit(MODE_PI2);
+
+template <int NT, uint32_t MODES>
 __global__ void __launch_bounds__(NT, 1)
 harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles, FastParams P) {
     constexpr int NW = NT / 32;
@@ -175,7 +191,7 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
         for (int p = 0; p < P.n_phases; ++p) {
             const PhaseDesc &ph = P.ph[p];
             const int n = ph.n_items;
-            if (ph.mode == MODE_CC) {
+            if ((MODES & bit(MODE_CC)) && ph.mode == MODE_CC) {
                 // lane -> (matrix row, 8-column half) of the 16x16 (or 16x8) operand tile
                 const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
                 if (ph.B == 16) {
@@ -205,7 +221,7 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
                         stmatrix_x2(addr, pack_bf16(c0[0], c0[1]), pack_bf16(c0[2], c0[3]));
                     }
                 }
-            } else if (ph.mode == MODE_SS && ph.B == 16) {
+            } else if ((MODES & bit(MODE_SS)) && ph.mode == MODE_SS && ph.B == 16) {
                 // software pipeline over this warp's items: operands of the next item are in
                 // flight while the current one is multiplied
                 uint4 rawA[4][2], rawB[4][2], bfA[8], bfB[8];
@@ -231,7 +247,7 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
                     ss16_store(c, ph, it2, rawB);
                     it = it3;
                 }
-            } else if (ph.mode == MODE_SS) {
+            } else if ((MODES & bit(MODE_SS)) && ph.mode == MODE_SS) {
                 const uint32_t *bf8 = reinterpret_cast<const uint32_t *>(ph.bfrag);
                 for (int it = warp; it < n; it += NW) {
                     const uint32_t a0 = c.sbase + 2u * (uint32_t)(c.g * pitch + c.q * ph.lane_step + tab_s[ph.items_off + it]);
@@ -252,7 +268,7 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
                         sts128(a1 + 2u * ph.j_off[j], raw[j][1]);
                     }
                 }
-            } else if (ph.mode == MODE_GS) {
+            } else if ((MODES & bit(MODE_GS)) && ph.mode == MODE_GS) {
                 uint4 rawA[4][2], rawB[4][2], bfA[8], bfB[8];
                 uint32_t mats[8][4];
                 int it = warp;
@@ -276,27 +292,25 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
                     gs_store(c, ph, it2, mats);
                     it = it3;
                 }
-            } else if (ph.mode == MODE_PO) {
-                // every operand of the phase is read before the barrier, every result is written
-                // after it; a warp owns at most two items: the first is multiplied before the
-                // barrier, the second only loaded
+            } else if ((MODES & bit(MODE_PO)) && ph.mode == MODE_PO) {
+                // contiguous blocks in (ldmatrix), eight-block runs out to the same sixteen 16-byte
+                // slots the item read (a per-item table names them): in place, no barrier
                 const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
-                const int it0 = warp, it1 = warp + NW;
-                uint4 out[4][2];
-                uint32_t a1[8][4];
-                if (it0 < n) {
-                    const int32_t *tab = tab_s + ph.items_off + it0 * 12;
+                for (int it = warp; it < n; it += NW) {
+                    const int32_t *tab = tab_s + ph.items_off + it * 24;
+                    uint4 bf[8], out[4][2];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) bf[e] = __ldg(ph.bfrag + (size_t)it * 256 + e * 32 + lane);
 #pragma unroll
                     for (int w = 0; w < 4; ++w) {
                         float acc[2][2][4];
 #pragma unroll
                         for (int ee = 0; ee < 2; ++ee) {
                             const int e = 2 * w + ee;
-                            const uint4 bf = __ldg(ph.bfrag + (size_t)it0 * 256 + e * 32 + lane);
                             uint32_t a[4];
                             ldmatrix_x4(a, c.sbase + 2u * (uint32_t)(mrow * pitch + tab[e] + mcol));
-                            mma_k16(acc[ee][0], a, bf.x, bf.y);
-                            mma_k16(acc[ee][1], a, bf.z, bf.w);
+                            mma_k16(acc[ee][0], a, bf[e].x, bf[e].y);
+                            mma_k16(acc[ee][1], a, bf[e].z, bf[e].w);
                         }
 #pragma unroll
                         for (int k = 0; k < 2; ++k)
@@ -306,50 +320,16 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
                                 for (int h = 0; h < 2; ++h)
                                     set_word(out[i + 2 * k][h], w, pack_bf16(acc[0][k][i + 2 * h], acc[1][k][i + 2 * h]));
                     }
-                }
-                if (it1 < n) {
-                    const int32_t *tab = tab_s + ph.items_off + it1 * 12;
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) ldmatrix_x4(a1[e], c.sbase + 2u * (uint32_t)(mrow * pitch + tab[e] + mcol));
-                }
-                __syncthreads();
-                if (it0 < n) {
-                    const uint32_t o0 = c.sbase + 2u * (uint32_t)(c.g * pitch + c.q * ph.lane_step + tab_s[ph.items_off + it0 * 12 + 8]);
-                    const uint32_t o1 = o0 + 2u * (uint32_t)(8 * pitch);
+                    // every lane's ldmatrix of this item precedes these stores in program order
+                    __syncwarp();
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        sts128(o0 + 2u * ph.j_off[j], out[j][0]);
-                        sts128(o1 + 2u * ph.j_off[j], out[j][1]);
+                        const uint32_t o0 = c.sbase + 2u * (uint32_t)(c.g * pitch + tab[8 + c.q + 4 * j]);
+                        sts128(o0, out[j][0]);
+                        sts128(o0 + 2u * (uint32_t)(8 * pitch), out[j][1]);
                     }
                 }
-                if (it1 < n) {
-#pragma unroll
-                    for (int w = 0; w < 4; ++w) {
-                        float acc[2][2][4];
-#pragma unroll
-                        for (int ee = 0; ee < 2; ++ee) {
-                            const int e = 2 * w + ee;
-                            const uint4 bf = __ldg(ph.bfrag + (size_t)it1 * 256 + e * 32 + lane);
-                            mma_k16(acc[ee][0], a1[e], bf.x, bf.y);
-                            mma_k16(acc[ee][1], a1[e], bf.z, bf.w);
-                        }
-#pragma unroll
-                        for (int k = 0; k < 2; ++k)
-#pragma unroll
-                            for (int i = 0; i < 2; ++i)
-#pragma unroll
-                                for (int h = 0; h < 2; ++h)
-                                    set_word(out[i + 2 * k][h], w, pack_bf16(acc[0][k][i + 2 * h], acc[1][k][i + 2 * h]));
-                    }
-                    const uint32_t o0 = c.sbase + 2u * (uint32_t)(c.g * pitch + c.q * ph.lane_step + tab_s[ph.items_off + it1 * 12 + 8]);
-                    const uint32_t o1 = o0 + 2u * (uint32_t)(8 * pitch);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        sts128(o0 + 2u * ph.j_off[j], out[j][0]);
-                        sts128(o1 + 2u * ph.j_off[j], out[j][1]);
-                    }
-                }
-            } else if (ph.mode == MODE_PI) {
+            } else if ((MODES & bit(MODE_PI)) && ph.mode == MODE_PI) {
                 const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
                 const int it0 = warp, it1 = warp + NW;
                 uint32_t mats[8][4];
@@ -393,7 +373,29 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
                     for (int e = 0; e < 8; ++e)
                         stmatrix_x4(c.sbase + 2u * (uint32_t)(mrow * pitch + tab[e] + mcol), mats[e][0], mats[e][1], mats[e][2], mats[e][3]);
                 }
-            } else {   // MODE_CG: operands from contiguous smem blocks, results scattered to global memory
+            } else if ((MODES & bit(MODE_PI2)) && ph.mode == MODE_PI2) {
+                // the reverse: sixteen slots in (eight-block runs), contiguous blocks out (stmatrix)
+                // to the same slots
+                const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
+                for (int it = warp; it < n; it += NW) {
+                    const int32_t *tab = tab_s + ph.items_off + it * 24;
+                    uint4 raw[4][2], bf[8];
+                    uint32_t mats[8][4];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) bf[e] = __ldg(ph.bfrag + (size_t)it * 256 + e * 32 + lane);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t i0 = c.sbase + 2u * (uint32_t)(c.g * pitch + tab[8 + c.q + 4 * j]);
+                        raw[j][0] = lds128(i0);
+                        raw[j][1] = lds128(i0 + 2u * (uint32_t)(8 * pitch));
+                    }
+                    octet_mma16<false>(raw, bf, mats);
+                    __syncwarp();
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        stmatrix_x4(c.sbase + 2u * (uint32_t)(mrow * pitch + tab[e] + mcol), mats[e][0], mats[e][1], mats[e][2], mats[e][3]);
+                }
+            } else if ((MODES & bit(MODE_CG)) && ph.mode == MODE_CG) {   // operands from contiguous smem blocks, results scattered to global memory
                 const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
                 for (int it = warp; it < n; it += NW) {
                     const int32_t *tab = tab_s + ph.items_off + it * 24;
@@ -453,6 +455,7 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
 struct FastPlan {
     FastParams fwd{}, bwd{};
     size_t smem_bytes = 0;
+    int variant_fwd = 0, variant_bwd = 0;     // which compiled set of phase modes each direction needs
     std::vector<void *> dev_allocs;
     int max_ctas = 0;
 };
@@ -508,7 +511,6 @@ harp_status_t harp_fast_build(harp_plan *plan) {
             }
             digitrev = plan->h_perm[(size_t)i] == src;
         }
-        if (d / 16 / 8 > 2 * (kThreads / 32)) digitrev = false;      // a warp holds at most two items over the barrier
     }
     std::vector<int64_t> inv;                                        // source coordinate -> natural coordinate
     if (!identity) {
@@ -518,31 +520,58 @@ harp_status_t harp_fast_build(harp_plan *plan) {
 
     // ---- shared-memory layouts.  "nat": coordinates in the plan's own order; "src": in the
     // order of the rows in global memory before the gather (digit-reversal scheme only).
-    // A layout gives every phase's local index an element stride W with W/8 mod 8 not in {0,4}.
+    // Local index r of a phase sits at element offset r*W + (r/4)*gp.  The four lanes q of a
+    // quarter-warp hold local indices lm*q + const, lm*W (+ gp when lm = 4) elements apart; that
+    // distance should be 2 or 6 (mod 8) 16-byte slots, which together with the odd row pitch puts
+    // the eight accesses of a quarter-warp into eight bank groups.  The strides also decide how
+    // the chunk copies of the tile hit the banks.  W (padding), gp (gap after every fourth step)
+    // and lm are chosen per phase by coordinate descent on the number of shared-memory wavefronts
+    // of the strided phases and of the two tile copies.
     struct Layout {
-        std::vector<int64_t> S, W;      // per phase: coordinate stride and shared-memory stride
-        std::vector<int> lm;            // per phase: lane multiplier (1 or 2)
+        std::vector<int64_t> S, W, gp;  // per phase: coordinate stride, shared-memory stride, gap
+        std::vector<int> lm;            // per phase: lane multiplier (1, 2 or 4)
         int64_t extent = 0;
+        int64_t off(int p, int64_t r) const { return r * W[(size_t)p] + (r / 4) * gp[(size_t)p]; }
     };
-    auto make_layout = [&](const std::vector<int> &order, const std::vector<int64_t> &strides) {
-        Layout L;
+    struct Choice { int pad, gap, lm; };                 // pad and gap in 16-byte slots
+    auto make_layout = [&](const std::vector<int> &order, const std::vector<int64_t> &strides,
+                           const std::vector<Choice> &ch, Layout &L) {
         L.S = strides;
         L.W.assign((size_t)np, 0);
+        L.gp.assign((size_t)np, 0);
         L.lm.assign((size_t)np, 1);
         int64_t W = 1;
         bool first = true;
         for (int p : order) {
+            const int B = phases[(size_t)p].B;
+            const Choice &c = ch[(size_t)p];
+            int64_t gp = 0;
             if (!first) {
-                W = (W + 7) / 8 * 8;
-                while (((W / 8) % 8) == 0 || ((W / 8) % 8) == 4) W += 8;
-                L.lm[(size_t)p] = ((W / 8) % 2 == 0) ? 1 : 2;
+                W = (W + 7) / 8 * 8 + 8 * c.pad;
+                gp = 8 * c.gap;
+                if (c.lm == 4 && B != 16) return false;
+                if (c.lm == 2 && gp != 0) return false;  // the lanes' slots would straddle a gap
+                L.lm[(size_t)p] = c.lm;
+            } else if (c.pad || c.gap || c.lm != 1) {
+                return false;
             }
             first = false;
             L.W[(size_t)p] = W;
-            W *= phases[(size_t)p].B;
+            L.gp[(size_t)p] = gp;
+            W = W * B + (B / 4 - 1) * gp;
         }
         L.extent = W;
-        return L;
+        return true;
+    };
+    auto pitch_of = [&](const Layout &L) {
+        int64_t pt = (L.extent + 7) / 8 * 8;
+        if ((pt / 8) % 2 == 0) pt += 8;
+        return pt;
+    };
+    auto worst_bank = [](const std::vector<int64_t> &slots) {   // wavefronts of one quarter-warp access
+        int cnt[8] = {0, 0, 0, 0, 0, 0, 0, 0}, worst = 0;
+        for (int64_t s : slots) worst = std::max(worst, ++cnt[((s % 8) + 8) % 8]);
+        return worst;
     };
     std::vector<int> order_nat((size_t)np), order_src((size_t)np);
     std::vector<int64_t> S_nat((size_t)np), S_src((size_t)np);
@@ -552,10 +581,129 @@ harp_status_t harp_fast_build(harp_plan *plan) {
         S_nat[(size_t)p] = phases[(size_t)p].S;
         S_src[(size_t)p] = d / (phases[(size_t)p].S * phases[(size_t)p].B);   // prod of radices above the phase
     }
-    const Layout Lnat = make_layout(order_nat, S_nat);
-    const Layout Lsrc = digitrev ? make_layout(order_src, S_src) : Lnat;
-    int64_t pitch = (std::max(Lnat.extent, Lsrc.extent) + 7) / 8 * 8;
-    if ((pitch / 8) % 2 == 0) pitch += 8;
+    // offset of a coordinate in a layout (coordinate in the layout's own order)
+    auto phys_in = [&](const Layout &L, int64_t pos) {
+        int64_t o = 0;
+        for (int p = 0; p < np; ++p) o += L.off(p, (pos / L.S[(size_t)p]) % phases[(size_t)p].B);
+        return o;
+    };
+    // In the digit-reversal scheme the output-ordered chunk map follows from the source layout:
+    // chunk (hi + lo + r*S)/8 of the output lives in slot (e, h) = (r & 7, r >> 3) of the item's
+    // eight source blocks (see reorder_slots below).
+    auto reorder_off = [&](const Layout &L, int64_t hi, int64_t lo, int sl) {
+        return phys_in(L, plan->h_perm[(size_t)(hi + lo + (sl & 7))]) + 8 * (sl >> 3);
+    };
+    auto layout_cost = [&](const Layout &L, bool src_scheme) {
+        const int64_t pc = pitch_of(L) / 8;
+        double cost = 1e-7 * (double)L.extent;
+        // strided phases: lanes q = 0..3 of two neighbouring rows
+        const std::vector<int> &order = src_scheme ? order_src : order_nat;
+        for (size_t k = 1; k < order.size(); ++k) {
+            const int p = order[k];
+            const int64_t step = L.lm[(size_t)p] * L.W[(size_t)p] + (L.lm[(size_t)p] == 4 ? L.gp[(size_t)p] : 0);
+            std::vector<int64_t> slots;
+            for (int q = 0; q < 4; ++q)
+                for (int row = 0; row < 2; ++row) slots.push_back(q * step / 8 + row * pc);
+            cost += 2.0 * worst_bank(slots);
+        }
+        // tile copies: eight neighbouring chunks of one row per quarter-warp
+        auto map_cost = [&](auto loc) {
+            double sum = 0;
+            for (int64_t c0 = 0; c0 < d / 8; c0 += 8) {
+                std::vector<int64_t> slots;
+                for (int64_t c = c0; c < std::min(d / 8, c0 + 8); ++c) slots.push_back(loc(c) / 8);
+                sum += worst_bank(slots);
+            }
+            return sum / (double)((d / 8 + 7) / 8);
+        };
+        cost += map_cost([&](int64_t c) { return phys_in(L, 8 * c); });
+        if (src_scheme) {
+            const HostPhase &hp = phases[(size_t)np - 1];
+            cost += map_cost([&](int64_t c) {
+                const int64_t o = 8 * c, span = hp.S * hp.B;                         // o = hi + lo + r*S
+                return reorder_off(L, o / span * span, o % hp.S, (int)((o / hp.S) % hp.B));
+            });
+        } else {
+            cost += map_cost([&](int64_t c) { return phys_in(L, 8 * c); });
+        }
+        return cost;
+    };
+    auto search_layout = [&](const std::vector<int> &order, const std::vector<int64_t> &strides, bool src_scheme, Layout &best) {
+        // start: the smallest padding that makes every strided phase conflict-free on its own
+        std::vector<Choice> ch((size_t)np, Choice{0, 0, 1});
+        {
+            int64_t W = 1;
+            bool first = true;
+            for (int p : order) {
+                if (!first) {
+                    W = (W + 7) / 8 * 8;
+                    int pad = 0;
+                    while (((W / 8 + pad) % 8) == 0 || ((W / 8 + pad) % 8) == 4) ++pad;
+                    ch[(size_t)p] = Choice{pad, 0, ((W / 8 + pad) % 2 == 0) ? 1 : 2};
+                    W += 8 * pad;
+                }
+                first = false;
+                W *= phases[(size_t)p].B;
+            }
+        }
+        if (!make_layout(order, strides, ch, best)) return false;
+        double best_cost = layout_cost(best, src_scheme);
+        if (order.size() == 3) {
+            // two free phases: try every pair of choices
+            const int p1 = order[1], p2 = order[2];
+            for (int c1 = 0; c1 < 96; ++c1)
+                for (int c2 = 0; c2 < 96; ++c2) {
+                    std::vector<Choice> trial = ch;
+                    trial[(size_t)p1] = Choice{c1 % 8, (c1 / 8) % 4, 1 << (c1 / 32)};
+                    trial[(size_t)p2] = Choice{c2 % 8, (c2 / 8) % 4, 1 << (c2 / 32)};
+                    Layout L;
+                    if (!make_layout(order, strides, trial, L)) continue;
+                    if ((size_t)kTileRows * pitch_of(L) * 2 > 200u * 1024u) continue;
+                    // skip layouts whose strided phases are not conflict-free on their own
+                    bool clean = true;
+                    const int64_t pc = pitch_of(L) / 8;
+                    for (int p : {p1, p2}) {
+                        const int64_t step = L.lm[(size_t)p] * L.W[(size_t)p] + (L.lm[(size_t)p] == 4 ? L.gp[(size_t)p] : 0);
+                        std::vector<int64_t> slots;
+                        for (int q = 0; q < 4; ++q)
+                            for (int row = 0; row < 2; ++row) slots.push_back(q * step / 8 + row * pc);
+                        clean = clean && worst_bank(slots) == 1;
+                    }
+                    if (!clean) continue;
+                    const double c = layout_cost(L, src_scheme);
+                    if (c < best_cost - 1e-12) { best_cost = c; best = L; ch = trial; }
+                }
+            return true;
+        }
+        for (int sweep = 0; sweep < 3; ++sweep) {
+            bool improved = false;
+            for (size_t k = 1; k < order.size(); ++k) {
+                const int p = order[k];
+                for (int pad = 0; pad < 8; ++pad)
+                    for (int gap = 0; gap < 4; ++gap)
+                        for (int lm = 1; lm <= 4; lm *= 2) {
+                            std::vector<Choice> trial = ch;
+                            trial[(size_t)p] = Choice{pad, gap, lm};
+                            Layout L;
+                            if (!make_layout(order, strides, trial, L)) continue;
+                            if ((size_t)kTileRows * pitch_of(L) * 2 > 200u * 1024u) continue;
+                            const double c = layout_cost(L, src_scheme);
+                            if (c < best_cost - 1e-12) { best_cost = c; best = L; ch = trial; improved = true; }
+                        }
+            }
+            if (!improved) break;
+        }
+        return true;
+    };
+    Layout Lnat, Lsrc;
+    if (!search_layout(order_nat, S_nat, false, Lnat)) return HARP_ERR_UNSUPPORTED;
+    if (digitrev) {
+        if (!search_layout(order_src, S_src, true, Lsrc)) return HARP_ERR_UNSUPPORTED;
+    } else {
+        Lsrc = Lnat;
+    }
+    // (the transpose direction of the digit-reversal scheme also uses the output-ordered layout)
+    int64_t pitch = std::max(pitch_of(Lsrc), pitch_of(Lnat));
     const size_t tile_bytes = (size_t)kTileRows * pitch * 2;
     if (tile_bytes > 227u * 1024u) return HARP_ERR_UNSUPPORTED;
 
@@ -571,18 +719,10 @@ harp_status_t harp_fast_build(harp_plan *plan) {
         }
         return r;
     };
-    auto phys_nat = [&](int64_t pos) {
-        int64_t o = 0;
-        for (int p = 0; p < np; ++p) o += ((pos / Lnat.S[(size_t)p]) % phases[(size_t)p].B) * Lnat.W[(size_t)p];
-        return o;
-    };
+    auto phys_nat = [&](int64_t pos) { return phys_in(Lnat, pos); };
     // source coordinate j: its phase-p source-local index is (j / S_src[p]) % B_p, written with the
     // group's digits reversed; the layout only needs that index
-    auto phys_src = [&](int64_t j) {
-        int64_t o = 0;
-        for (int p = 0; p < np; ++p) o += ((j / Lsrc.S[(size_t)p]) % phases[(size_t)p].B) * Lsrc.W[(size_t)p];
-        return o;
-    };
+    auto phys_src = [&](int64_t j) { return phys_in(Lsrc, j); };
 
     // ---- first-phase octets for the global gather/scatter scheme
     const int B0 = phases[0].B;
@@ -615,13 +755,36 @@ harp_status_t harp_fast_build(harp_plan *plan) {
         chunk_nat[(size_t)c] = (int32_t)phys_nat(8 * c);
         chunk_src[(size_t)c] = (int32_t)phys_src(8 * c);
     }
+    const std::vector<int32_t> chunk_nat_plain(chunk_nat);   // output order in the output-ordered layout
+    // Digit reversal: the phase next to the output reorders the tile in place.  An item is eight
+    // blocks that are neighbours in output order; each is 16 contiguous source coordinates, so the
+    // item owns sixteen 16-byte slots of the source-ordered layout.  After the phase slot
+    // (e, h) = (r & 7, r >> 3) holds, for output local index r, the eight blocks' values: a run
+    // of eight neighbouring output coordinates.  reorder_slots[item][r] is that slot's offset, and
+    // the output-ordered chunk map follows from it.
+    std::vector<int32_t> reorder_slots;
+    if (digitrev) {
+        const HostPhase &hp = phases[(size_t)np - 1];
+        const int64_t span = hp.S * hp.B;
+        for (int64_t hi = 0; hi < d; hi += span)
+            for (int64_t lo = 0; lo < hp.S; lo += 8)
+                for (int r = 0; r < 16; ++r) {
+                    const int32_t off = (int32_t)reorder_off(Lsrc, hi, lo, r);
+                    reorder_slots.push_back(off);
+                    chunk_nat[(size_t)((hi + lo + (int64_t)r * hp.S) / 8)] = off;
+                }
+    }
+
+    // digit reversal, transpose direction: the barrier variant of the reordering phase (a warp
+    // holds at most two items over the barrier) measures faster than the in-place one
+    const bool pi_barrier = digitrev && d / 16 / 8 <= 2 * (kThreads / 32);
 
     auto sign_v = [&](int64_t i) -> double {             // sign seen by coordinate i after the gather
         if (plan->h_signs.empty()) return 1.0;
         const int64_t src = identity ? i : plan->h_perm[(size_t)i];
         return (double)plan->h_signs[(size_t)src];
     };
-    static const int joff1_16[4] = {0, 4, 8, 12}, joff2_16[4] = {0, 1, 8, 9};
+    static const int joff1_16[4] = {0, 4, 8, 12}, joff2_16[4] = {0, 1, 8, 9}, joff4_16[4] = {0, 1, 2, 3};
     static const int joff1_8[4] = {0, 4, 0, 0}, joff2_8[4] = {0, 1, 0, 0};
 
     for (int dir = 0; dir < 2 && st == HARP_OK; ++dir) {  // 0 = forward, 1 = transpose
@@ -629,15 +792,19 @@ harp_status_t harp_fast_build(harp_plan *plan) {
         P.n_phases = np;
         P.d = (int32_t)d;
         P.pitch = (int32_t)pitch;
+        // chunk maps: output order (for the digit-reversal scheme: where the in-place reordering
+        // phase leaves / expects it), source order, and output order in the output-ordered layout
         std::vector<int32_t> tables(chunk_nat);
         const int32_t off_nat = 0;
         const int32_t off_src = (int32_t)tables.size();
         tables.insert(tables.end(), chunk_src.begin(), chunk_src.end());
+        const int32_t off_natl = (int32_t)tables.size();
+        if (digitrev && pi_barrier) tables.insert(tables.end(), chunk_nat_plain.begin(), chunk_nat_plain.end());
         if (identity) {
             P.copy_in = off_nat;
             P.copy_out = off_nat;
         } else if (digitrev) {
-            P.copy_in = dir == 0 ? off_src : off_nat;
+            P.copy_in = dir == 0 ? off_src : (pi_barrier ? off_natl : off_nat);
             P.copy_out = dir == 0 ? off_nat : off_src;
         } else {
             P.copy_in = dir == 0 ? -1 : off_nat;
@@ -650,21 +817,23 @@ harp_status_t harp_fast_build(harp_plan *plan) {
             const int B = hp.B;
             int mode;
             if (identity) mode = p == 0 ? MODE_CC : MODE_SS;
-            else if (digitrev) mode = p == np - 1 ? (dir == 0 ? MODE_PO : MODE_PI) : MODE_SS;
+            else if (digitrev) mode = p == np - 1 ? (dir == 0 ? MODE_PO : (pi_barrier ? MODE_PI : MODE_PI2)) : MODE_SS;
             else mode = p == 0 ? (dir == 0 ? MODE_GS : MODE_CG) : MODE_SS;
             D.mode = mode;
             D.B = B;
             // Which layout do the strided accesses of this phase use, and with which slot geometry?
             const bool src_side = digitrev && mode == MODE_SS;          // in place on the source-ordered layout
             const Layout &L = src_side ? Lsrc : Lnat;
-            const int lm = (mode == MODE_GS || mode == MODE_CG || mode == MODE_CC) ? 1 : L.lm[(size_t)p];
-            const int *jo = B == 16 ? (lm == 1 ? joff1_16 : joff2_16) : (lm == 1 ? joff1_8 : joff2_8);
+            const int lm = (mode == MODE_GS || mode == MODE_CG || mode == MODE_CC || mode == MODE_PO || mode == MODE_PI2)
+                               ? 1 : L.lm[(size_t)p];   // table-indexed slots use the plain map
+            const int *jo = B == 16 ? (lm == 1 ? joff1_16 : lm == 2 ? joff2_16 : joff4_16) : (lm == 1 ? joff1_8 : joff2_8);
             if (mode == MODE_GS || mode == MODE_CG) {    // these index the item table by slot
                 D.lane_step = lm;
                 for (int j = 0; j < 4; ++j) D.j_off[j] = jo[j];
             } else {
-                D.lane_step = (int32_t)(lm * L.W[(size_t)p]);
-                for (int j = 0; j < 4; ++j) D.j_off[j] = (int32_t)(jo[j] * L.W[(size_t)p]);
+                // the slots of one lane group never straddle a gap: q*lm steps with lm = 4, j steps otherwise
+                D.lane_step = (int32_t)(lm * L.W[(size_t)p] + (lm == 4 ? L.gp[(size_t)p] : 0));
+                for (int j = 0; j < 4; ++j) D.j_off[j] = (int32_t)L.off(p, jo[j]);
             }
             // local index seen by the strided / contiguous side of the operand, as a natural local index
             auto strided_nat = [&](int slot) {
@@ -672,7 +841,7 @@ harp_status_t harp_fast_build(harp_plan *plan) {
                 return src_side ? nat_local_of_src_local(p, r) : r;
             };
             auto contig_nat = [&](int slot) {            // contiguous blocks of PO/PI live in the source layout
-                return (mode == MODE_PO || mode == MODE_PI) ? nat_local_of_src_local(p, slot) : slot;
+                return (mode == MODE_PO || mode == MODE_PI || mode == MODE_PI2) ? nat_local_of_src_local(p, slot) : slot;
             };
             // enumerate items and the natural base coordinate of every block
             std::vector<int32_t> items;
@@ -698,9 +867,8 @@ harp_status_t harp_fast_build(harp_plan *plan) {
                         items.push_back((int32_t)phys_src(hi + lo));
                         for (int e = 0; e < 8; ++e) block_base.push_back(inv[(size_t)(hi + lo + e)]);
                     }
-            } else if (mode == MODE_PO || mode == MODE_PI) {
-                // octets of blocks that are neighbours in natural order; each block is 16 contiguous
-                // source coordinates
+            } else if (mode == MODE_PI) {
+                // as below, but the strided side lives in the output-ordered layout
                 ints_per_item = 12;
                 const int64_t span = hp.S * B;
                 for (int64_t hi = 0; hi < d; hi += span)
@@ -711,6 +879,20 @@ harp_status_t harp_fast_build(harp_plan *plan) {
                         }
                         items.push_back((int32_t)phys_nat(hi + lo));
                         items.push_back(0); items.push_back(0); items.push_back(0);
+                    }
+            } else if (mode == MODE_PO || mode == MODE_PI2) {
+                // octets of blocks that are neighbours in natural order; each block is 16 contiguous
+                // source coordinates
+                ints_per_item = 24;
+                const int64_t span = hp.S * B;
+                size_t item_no = 0;
+                for (int64_t hi = 0; hi < d; hi += span)
+                    for (int64_t lo = 0; lo < hp.S; lo += 8, ++item_no) {
+                        for (int e = 0; e < 8; ++e) {
+                            items.push_back((int32_t)phys_src(plan->h_perm[(size_t)(hi + lo + e)]));
+                            block_base.push_back(hi + lo + e);
+                        }
+                        for (int r = 0; r < 16; ++r) items.push_back(reorder_slots[item_no * 16 + (size_t)r]);
                     }
             } else {
                 ints_per_item = 24;
@@ -741,11 +923,17 @@ harp_status_t harp_fast_build(harp_plan *plan) {
                     for (int32_t b : items) ok = ok && contig_ok(b);
                 } else if (mode == MODE_SS) {
                     for (int32_t b : items) ok = ok && strided_ok(b);
-                } else if (mode == MODE_PO || mode == MODE_PI) {
+                } else if (mode == MODE_PI) {
                     ok = ok && B == 16 && D.n_items <= 2 * (kThreads / 32);
                     for (size_t i = 0; i < items.size(); i += 12) {
                         for (int e = 0; e < 8; ++e) ok = ok && contig_ok(items[i + e]);
                         ok = ok && strided_ok(items[i + 8]);
+                    }
+                } else if (mode == MODE_PO || mode == MODE_PI2) {
+                    ok = ok && B == 16 && hp.S % 8 == 0;
+                    for (size_t i = 0; i < items.size(); i += 24) {
+                        for (int e = 0; e < 8; ++e) ok = ok && contig_ok(items[i + e]);
+                        for (int r = 0; r < 16; ++r) ok = ok && items[i + 8 + r] >= 0 && items[i + 8 + r] % 8 == 0 && items[i + 8 + r] + 8 <= pitch;
                     }
                 } else {
                     for (size_t i = 0; i < items.size(); i += 24) {
@@ -758,7 +946,7 @@ harp_status_t harp_fast_build(harp_plan *plan) {
             D.items_off = (int32_t)tables.size();
             tables.insert(tables.end(), items.begin(), items.end());
             // fragments: B[k-slot][n-slot] = G[local index of the k-slot][local index of the n-slot]
-            const bool in_strided = (mode == MODE_SS || mode == MODE_GS || mode == MODE_PI);
+            const bool in_strided = (mode == MODE_SS || mode == MODE_GS || mode == MODE_PI || mode == MODE_PI2);
             const bool out_strided = (mode == MODE_SS || mode == MODE_CG || mode == MODE_PO);
             const int words_per_lane = B == 16 ? 4 : 1;
             std::vector<uint32_t> frag(block_base.size() * 32 * words_per_lane);
@@ -799,8 +987,13 @@ harp_status_t harp_fast_build(harp_plan *plan) {
     }
     if (st == HARP_OK && fp->smem_bytes > 227u * 1024u) st = HARP_ERR_UNSUPPORTED;
     if (st == HARP_OK) {
-        if (cudaFuncSetAttribute(harp_fast_kernel<kThreads>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+        if (cudaFuncSetAttribute(harp_fast_kernel<kThreads, kModesGeneral>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(harp_fast_kernel<kThreads, kModesReorderOut>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(harp_fast_kernel<kThreads, kModesReorderIn>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+            cudaFuncSetAttribute(harp_fast_kernel<kThreads, kModesReorderIn2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
             st = HARP_ERR_CUDA;
+        fp->variant_fwd = digitrev ? 1 : 0;
+        fp->variant_bwd = digitrev ? (pi_barrier ? 2 : 3) : 0;
         int dev = 0, sms = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -829,8 +1022,14 @@ harp_status_t harp_fast_apply(const harp_plan *plan, void *x, int64_t n_rows, ha
     if ((reinterpret_cast<uintptr_t>(x) & 15u) != 0) return HARP_ERR_UNSUPPORTED;
     const int64_t n_tiles = (n_rows + kTileRows - 1) / kTileRows;
     const int grid = (int)std::min<int64_t>(n_tiles, fp->max_ctas);
-    harp_fast_kernel<kThreads><<<grid, kThreads, fp->smem_bytes, stream>>>(static_cast<__nv_bfloat16 *>(x), n_rows, n_tiles,
-                                                                 transpose ? fp->bwd : fp->fwd);
+    __nv_bfloat16 *xb = static_cast<__nv_bfloat16 *>(x);
+    const FastParams &P = transpose ? fp->bwd : fp->fwd;
+    switch (transpose ? fp->variant_bwd : fp->variant_fwd) {
+        case 1: harp_fast_kernel<kThreads, kModesReorderOut><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, P); break;
+        case 2: harp_fast_kernel<kThreads, kModesReorderIn><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, P); break;
+        case 3: harp_fast_kernel<kThreads, kModesReorderIn2><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, P); break;
+        default: harp_fast_kernel<kThreads, kModesGeneral><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, P); break;
+    }
     g_harp_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HARP_OK : HARP_ERR_CUDA;
 }

@@ -14,7 +14,7 @@ struct HostPhase {
     int B;               // fused block size
     int64_t S;           // natural stride of the phase (= s_{t0})
     int64_t W;           // shared-memory element stride of the phase's local index
-    int lane_mult;       // 1 or 2
+    int lane_mult;       // 1, 2 or (B = 16 only) 4
 };
 
 inline uint16_t f2bf(double v) {
@@ -59,8 +59,8 @@ inline int strided_slot(int kappa, int B, int lane_mult) {
     const int qq = (kappa & 7) >> 1, i = kappa & 1, k = kappa >> 3;
     const int j = i + 2 * k;
     if (B == 16) {
-        static const int joff1[4] = {0, 4, 8, 12}, joff2[4] = {0, 1, 8, 9};
-        return lane_mult * qq + (lane_mult == 1 ? joff1[j] : joff2[j]);
+        static const int joff1[4] = {0, 4, 8, 12}, joff2[4] = {0, 1, 8, 9}, joff4[4] = {0, 1, 2, 3};
+        return lane_mult * qq + (lane_mult == 1 ? joff1[j] : lane_mult == 2 ? joff2[j] : joff4[j]);
     }
     static const int joff1[2] = {0, 4}, joff2[2] = {0, 1};
     return lane_mult * qq + (lane_mult == 1 ? joff1[j] : joff2[j]);
