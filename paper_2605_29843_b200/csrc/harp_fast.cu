@@ -759,17 +759,43 @@ harp_status_t harp_fast_build(harp_plan *plan) {
     // Digit reversal: the phase next to the output reorders the tile in place.  An item is eight
     // blocks that are neighbours in output order; each is 16 contiguous source coordinates, so the
     // item owns sixteen 16-byte slots of the source-ordered layout.  After the phase slot
-    // (e, h) = (r & 7, r >> 3) holds, for output local index r, the eight blocks' values: a run
-    // of eight neighbouring output coordinates.  reorder_slots[item][r] is that slot's offset, and
-    // the output-ordered chunk map follows from it.
+    // (e, h) = (s & 7, s >> 3), s = slot_of[r], holds, for output local index r, the eight blocks'
+    // values: a run of eight neighbouring output coordinates.  reorder_slots[item][r] is that
+    // slot's offset, and the output-ordered chunk map follows from it.
     std::vector<int32_t> reorder_slots;
     if (digitrev) {
         const HostPhase &hp = phases[(size_t)np - 1];
         const int64_t span = hp.S * hp.B;
+        // The four lanes q of a quarter-warp access the slots of r = q + 4j in two neighbouring
+        // rows.  Starting from the identity, swap pairs while that lowers the number of
+        // shared-memory wavefronts (judged on the first item; the other items differ by a
+        // constant offset).
+        int slot_of[16];
+        for (int r = 0; r < 16; ++r) slot_of[r] = r;
+        auto slot_cost = [&]() {
+            int total = 0;
+            for (int j = 0; j < 4; ++j) {
+                std::vector<int64_t> slots;
+                for (int q = 0; q < 4; ++q)
+                    for (int row = 0; row < 2; ++row) slots.push_back(reorder_off(Lsrc, 0, 0, slot_of[q + 4 * j]) / 8 + row * (pitch / 8));
+                total += worst_bank(slots);
+            }
+            return total;
+        };
+        for (bool improved = true; improved;) {
+            improved = false;
+            for (int a = 0; a < 16; ++a)
+                for (int b = a + 1; b < 16; ++b) {
+                    const int before = slot_cost();
+                    std::swap(slot_of[a], slot_of[b]);
+                    if (slot_cost() < before) improved = true;
+                    else std::swap(slot_of[a], slot_of[b]);
+                }
+        }
         for (int64_t hi = 0; hi < d; hi += span)
             for (int64_t lo = 0; lo < hp.S; lo += 8)
                 for (int r = 0; r < 16; ++r) {
-                    const int32_t off = (int32_t)reorder_off(Lsrc, hi, lo, r);
+                    const int32_t off = (int32_t)reorder_off(Lsrc, hi, lo, slot_of[r]);
                     reorder_slots.push_back(off);
                     chunk_nat[(size_t)((hi + lo + (int64_t)r * hp.S) / 8)] = off;
                 }
