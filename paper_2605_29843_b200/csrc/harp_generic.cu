@@ -105,12 +105,26 @@ harp_generic_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_cta, 
 // b x b kernel in registers and walks over the rows of the tile, so a block kernel is fetched
 // once per tile instead of once per output coordinate, all index arithmetic is done once per
 // block, and (a block being updated in place by its only owner) one barrier per stage suffices.
-template <int B>
+// Position of coordinate i of a row in shared memory.  With SWZ the index bits 2-4 are XORed with
+// bits 5-6 (inside aligned runs of 128 coordinates, so d must be a multiple of 128): the lanes
+// of a warp, which own neighbouring blocks, then read and write 32 different banks also in the
+// stages of stride 4 and 16, where the plain layout gives 4- and 2-way conflicts; aligned
+// groups of four coordinates stay together.
+template <bool SWZ>
+__device__ __forceinline__ int row_pos(int i) {
+    return SWZ ? (i ^ (((i >> 5) & 3) << 2) ^ (((i >> 6) & 1) << 4)) : i;
+}
+
+template <int B, bool SWZ>
 __device__ __forceinline__ void stage_blocks(float *v, int rows, int d, int s, const float *__restrict__ Kt, int transpose) {
     const int nblk = d / B;
     for (int c = threadIdx.x; c < nblk; c += blockDim.x) {
         const int alpha = c / s, beta = c - alpha * s;
-        float *p = v + alpha * B * s + beta;
+        const int base = alpha * B * s + beta;
+        int pos[B];
+#pragma unroll
+        for (int i = 0; i < B; ++i) pos[i] = row_pos<SWZ>(base + i * s);
+        float *p = v;
         float K[B][B];
         const float *Kc = Kt + (size_t)c * B * B;
         // a stage's block array starts at a multiple of 4 bytes only; the 16-byte load needs more
@@ -129,20 +143,32 @@ __device__ __forceinline__ void stage_blocks(float *v, int rows, int d, int s, c
 #pragma unroll 2
         for (int r = 0; r < rows; ++r, p += d) {
             float in[B];
+            if (B == 4 && s == 1) {              // the block is one aligned 16-byte group
+                const float4 q4 = *reinterpret_cast<const float4 *>(p + pos[0]);
+                in[0] = q4.x; in[1] = q4.y; in[2 % B] = q4.z; in[3 % B] = q4.w;
+            } else {
 #pragma unroll
-            for (int i = 0; i < B; ++i) in[i] = p[i * s];
+                for (int i = 0; i < B; ++i) in[i] = p[pos[i]];
+            }
+            float out[B];
 #pragma unroll
             for (int j = 0; j < B; ++j) {
                 float a = in[0] * K[0][j];
 #pragma unroll
                 for (int i = 1; i < B; ++i) a = fmaf(in[i], K[i][j], a);
-                p[j * s] = a;
+                out[j] = a;
+            }
+            if (B == 4 && s == 1) {
+                *reinterpret_cast<float4 *>(p + pos[0]) = make_float4(out[0], out[1], out[2 % B], out[3 % B]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < B; ++j) p[pos[j]] = out[j];
             }
         }
     }
 }
 
-template <typename T, int NT, bool BIG>
+template <typename T, int NT, bool BIG, bool SWZ>
 __global__ void __launch_bounds__(NT, 1)
 harp_blockowner_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_cta, StageTable st,
                        const float *__restrict__ blocks, const int32_t *__restrict__ perm,
@@ -157,21 +183,21 @@ harp_blockowner_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_ct
         const float sg = (!transpose && signs && signs[src] < 0) ? -1.f : 1.f;
         const T *col = xt + src;
 #pragma unroll 4
-        for (int r = 0; r < rows; ++r) v[r * d + i] = sg * to_f32<T>(col[(int64_t)r * d]);
+        for (int r = 0; r < rows; ++r) v[r * d + row_pos<SWZ>(i)] = sg * to_f32<T>(col[(int64_t)r * d]);
     }
     __syncthreads();
     for (int k = 0; k < st.m; ++k) {
         const int t = transpose ? st.m - 1 - k : k;
         const float *Kt = blocks + st.off[t];
         const int b = st.b[t];
-        if (b == 2) stage_blocks<2>(v, rows, d, st.s[t], Kt, transpose);
-        else if (b == 3) stage_blocks<3>(v, rows, d, st.s[t], Kt, transpose);
-        else if (b == 4) stage_blocks<4>(v, rows, d, st.s[t], Kt, transpose);
+        if (b == 2) stage_blocks<2, SWZ>(v, rows, d, st.s[t], Kt, transpose);
+        else if (b == 3) stage_blocks<3, SWZ>(v, rows, d, st.s[t], Kt, transpose);
+        else if (b == 4) stage_blocks<4, SWZ>(v, rows, d, st.s[t], Kt, transpose);
         else if (BIG) {
-            if (b == 5) stage_blocks<5>(v, rows, d, st.s[t], Kt, transpose);
-            else if (b == 6) stage_blocks<6>(v, rows, d, st.s[t], Kt, transpose);
-            else if (b == 7) stage_blocks<7>(v, rows, d, st.s[t], Kt, transpose);
-            else stage_blocks<8>(v, rows, d, st.s[t], Kt, transpose);
+            if (b == 5) stage_blocks<5, SWZ>(v, rows, d, st.s[t], Kt, transpose);
+            else if (b == 6) stage_blocks<6, SWZ>(v, rows, d, st.s[t], Kt, transpose);
+            else if (b == 7) stage_blocks<7, SWZ>(v, rows, d, st.s[t], Kt, transpose);
+            else stage_blocks<8, SWZ>(v, rows, d, st.s[t], Kt, transpose);
         }
         __syncthreads();
     }
@@ -181,14 +207,14 @@ harp_blockowner_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_ct
         const float sg = (transpose && signs && signs[dst] < 0) ? -1.f : 1.f;
         T *col = xt + dst;
 #pragma unroll 4
-        for (int r = 0; r < rows; ++r) col[(int64_t)r * d] = from_f32<T>(sg * v[r * d + i]);
+        for (int r = 0; r < rows; ++r) col[(int64_t)r * d] = from_f32<T>(sg * v[r * d + row_pos<SWZ>(i)]);
     }
 }
 
-template <typename T, int NT, bool BIG>
-harp_status_t launch_blockowner(const harp_plan *plan, const StageTable &st, const float *blocks, void *x, int64_t n_rows,
-                                int transpose, cudaStream_t stream) {
-    auto kern = harp_blockowner_kernel<T, NT, BIG>;
+template <typename T, int NT, bool BIG, bool SWZ>
+harp_status_t launch_blockowner_swz(const harp_plan *plan, const StageTable &st, const float *blocks, void *x, int64_t n_rows,
+                                    int transpose, cudaStream_t stream) {
+    auto kern = harp_blockowner_kernel<T, NT, BIG, SWZ>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
         return HARP_ERR_CUDA;
     int dev = 0, sms = 148;
@@ -206,6 +232,14 @@ harp_status_t launch_blockowner(const harp_plan *plan, const StageTable &st, con
                                                                               blocks, plan->d_perm, plan->d_signs, transpose);
     g_harp_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HARP_OK : HARP_ERR_CUDA;
+}
+
+template <typename T, int NT, bool BIG>
+harp_status_t launch_blockowner(const harp_plan *plan, const StageTable &st, const float *blocks, void *x, int64_t n_rows,
+                                int transpose, cudaStream_t stream) {
+    // the bank swizzle permutes inside aligned runs of 128 coordinates
+    return plan->d % 128 == 0 ? launch_blockowner_swz<T, NT, BIG, true>(plan, st, blocks, x, n_rows, transpose, stream)
+                              : launch_blockowner_swz<T, NT, BIG, false>(plan, st, blocks, x, n_rows, transpose, stream);
 }
 
 template <typename T, int ITEMS>
