@@ -21,6 +21,28 @@ constexpr int kMaxItems = 32;   // R*d <= kThreads*kMaxItems
 template <typename T> __device__ __forceinline__ float to_f32(T v);
 template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+// four neighbouring elements, p aligned to 4 * sizeof(T)
+template <typename T> __device__ __forceinline__ void load4(const T *p, float (&e)[4]);
+template <> __device__ __forceinline__ void load4<float>(const float *p, float (&e)[4]) {
+    const float4 q = *reinterpret_cast<const float4 *>(p);
+    e[0] = q.x; e[1] = q.y; e[2] = q.z; e[3] = q.w;
+}
+template <> __device__ __forceinline__ void load4<__nv_bfloat16>(const __nv_bfloat16 *p, float (&e)[4]) {
+    const uint2 q = *reinterpret_cast<const uint2 *>(p);
+    e[0] = __uint_as_float(q.x << 16); e[1] = __uint_as_float(q.x & 0xffff0000u);
+    e[2] = __uint_as_float(q.y << 16); e[3] = __uint_as_float(q.y & 0xffff0000u);
+}
+template <typename T> __device__ __forceinline__ void store4(T *p, const float (&e)[4]);
+template <> __device__ __forceinline__ void store4<float>(float *p, const float (&e)[4]) {
+    *reinterpret_cast<float4 *>(p) = make_float4(e[0], e[1], e[2], e[3]);
+}
+template <> __device__ __forceinline__ void store4<__nv_bfloat16>(__nv_bfloat16 *p, const float (&e)[4]) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(e[0], e[1]), hi = __floats2bfloat162_rn(e[2], e[3]);
+    uint2 q;
+    q.x = *reinterpret_cast<const uint32_t *>(&lo);
+    q.y = *reinterpret_cast<const uint32_t *>(&hi);
+    *reinterpret_cast<uint2 *>(p) = q;
+}
 template <typename T> __device__ __forceinline__ T from_f32(float v);
 template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
@@ -177,13 +199,32 @@ harp_blockowner_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_ct
     const int64_t row0 = (int64_t)blockIdx.x * rows_per_cta;
     const int rows = (int)min((int64_t)rows_per_cta, n_rows - row0);
     T *xt = x + row0 * d;
+    // without a permutation a thread moves aligned groups of four coordinates (one vector access in
+    // global and one in shared memory; the swizzle keeps such groups together)
+    const bool vec4 = !perm && d % 4 == 0 && (reinterpret_cast<uintptr_t>(x) % (4 * sizeof(T))) == 0;
     // a1-a3: load, sign, gather (forward) -- or plain load (transpose); a thread keeps its columns
-    for (int i = threadIdx.x; i < d; i += NT) {
-        const int src = (!transpose && perm) ? perm[i] : i;
-        const float sg = (!transpose && signs && signs[src] < 0) ? -1.f : 1.f;
-        const T *col = xt + src;
+    if (vec4) {
+        for (int i = 4 * threadIdx.x; i < d; i += 4 * NT) {
+            float sg[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) sg[k] = (!transpose && signs && signs[i + k] < 0) ? -1.f : 1.f;
+            const T *col = xt + i;
+            float *dst = v + row_pos<SWZ>(i);
 #pragma unroll 4
-        for (int r = 0; r < rows; ++r) v[r * d + row_pos<SWZ>(i)] = sg * to_f32<T>(col[(int64_t)r * d]);
+            for (int r = 0; r < rows; ++r) {
+                float e[4];
+                load4<T>(col + (int64_t)r * d, e);
+                *reinterpret_cast<float4 *>(dst + r * d) = make_float4(sg[0] * e[0], sg[1] * e[1], sg[2] * e[2], sg[3] * e[3]);
+            }
+        }
+    } else {
+        for (int i = threadIdx.x; i < d; i += NT) {
+            const int src = (!transpose && perm) ? perm[i] : i;
+            const float sg = (!transpose && signs && signs[src] < 0) ? -1.f : 1.f;
+            const T *col = xt + src;
+#pragma unroll 4
+            for (int r = 0; r < rows; ++r) v[r * d + row_pos<SWZ>(i)] = sg * to_f32<T>(col[(int64_t)r * d]);
+        }
     }
     __syncthreads();
     for (int k = 0; k < st.m; ++k) {
@@ -202,12 +243,28 @@ harp_blockowner_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_ct
         __syncthreads();
     }
     // a5: store -- or scatter and sign (transpose)
-    for (int i = threadIdx.x; i < d; i += NT) {
-        const int dst = (transpose && perm) ? perm[i] : i;
-        const float sg = (transpose && signs && signs[dst] < 0) ? -1.f : 1.f;
-        T *col = xt + dst;
+    if (vec4) {
+        for (int i = 4 * threadIdx.x; i < d; i += 4 * NT) {
+            float sg[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) sg[k] = (transpose && signs && signs[i + k] < 0) ? -1.f : 1.f;
+            T *col = xt + i;
+            const float *src = v + row_pos<SWZ>(i);
 #pragma unroll 4
-        for (int r = 0; r < rows; ++r) col[(int64_t)r * d] = from_f32<T>(sg * v[r * d + row_pos<SWZ>(i)]);
+            for (int r = 0; r < rows; ++r) {
+                const float4 q4 = *reinterpret_cast<const float4 *>(src + r * d);
+                const float e[4] = {sg[0] * q4.x, sg[1] * q4.y, sg[2] * q4.z, sg[3] * q4.w};
+                store4<T>(col + (int64_t)r * d, e);
+            }
+        }
+    } else {
+        for (int i = threadIdx.x; i < d; i += NT) {
+            const int dst = (transpose && perm) ? perm[i] : i;
+            const float sg = (transpose && signs && signs[dst] < 0) ? -1.f : 1.f;
+            T *col = xt + dst;
+#pragma unroll 4
+            for (int r = 0; r < rows; ++r) col[(int64_t)r * d] = from_f32<T>(sg * v[r * d + row_pos<SWZ>(i)]);
+        }
     }
 }
 
