@@ -155,6 +155,7 @@ extern "C" void harp_plan_destroy(harp_plan_t *p) {
         }
         if (p->d_blocks) cudaFree(p->d_blocks);
         if (p->d_fused_blocks) cudaFree(p->d_fused_blocks);
+        if (p->d_bo_blocks) cudaFree(p->d_bo_blocks);
         if (p->d_perm) cudaFree(p->d_perm);
         if (p->d_signs) cudaFree(p->d_signs);
     }

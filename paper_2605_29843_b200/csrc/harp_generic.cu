@@ -10,6 +10,8 @@
 // it applies.
 #include <algorithm>
 
+#include <cstdlib>
+
 #include "harp_internal.h"
 #include "harp_fuse.h"
 
@@ -148,20 +150,11 @@ __device__ __forceinline__ void stage_blocks(float *v, int rows, int d, int s, c
         for (int i = 0; i < B; ++i) pos[i] = row_pos<SWZ>(base + i * s);
         float *p = v;
         float K[B][B];
-        const float *Kc = Kt + (size_t)c * B * B;
-        // a stage's block array starts at a multiple of 4 bytes only; the 16-byte load needs more
-        if (B == 2 && (reinterpret_cast<uintptr_t>(Kt) & 15u) == 0) {
-            const float4 k4 = __ldg(reinterpret_cast<const float4 *>(Kc));
-            K[0][0] = k4.x;
-            K[0][1] = transpose ? k4.z : k4.y;
-            K[1][0] = transpose ? k4.y : k4.z;
-            K[1][1] = k4.w;
-        } else {
+        const float *Kc = Kt + c;                // element-major: entry k of block c at Kt[k * nblk + c]
 #pragma unroll
-            for (int i = 0; i < B; ++i)
+        for (int i = 0; i < B; ++i)
 #pragma unroll
-                for (int j = 0; j < B; ++j) K[i][j] = __ldg(Kc + (transpose ? j * B + i : i * B + j));
-        }
+            for (int j = 0; j < B; ++j) K[i][j] = __ldg(Kc + (size_t)(transpose ? j * B + i : i * B + j) * nblk);
 #pragma unroll 2
         for (int r = 0; r < rows; ++r, p += d) {
             float in[B];
@@ -299,6 +292,167 @@ harp_status_t launch_blockowner(const harp_plan *plan, const StageTable &st, con
                               : launch_blockowner_swz<T, NT, BIG, false>(plan, st, blocks, x, n_rows, transpose, stream);
 }
 
+// ---------------------------------------------------------------------------------------
+// Block-owner kernel on a transposed tile.  The tile is kept as [coordinate][row] with the row
+// index fastest, so a thread that owns a block reads and writes four rows of one coordinate with
+// one 16-byte access: a quarter of the shared-memory instructions of the row-major form, which is
+// bound by their issue rate.  Coordinate x lives at tpos(x) * R4 (R4 = padded row count, a
+// multiple of 4 with R4/4 odd): tpos XORs the low three index bits with bits 3 and 4 so that the
+// eight lanes of a quarter-warp -- eight neighbouring blocks of any stage, eight neighbouring
+// coordinates or coordinate quads in the copies -- fall into eight different bank groups
+// (needs d to be a multiple of 32).  The copies transpose 4 x 4 in registers.
+__device__ __forceinline__ int tpos(int x) { return x ^ (((x >> 4) & 1) * 5) ^ (((x >> 3) & 1) * 2); }
+
+__device__ __forceinline__ float4 f4_scale(float4 a, float k) { return make_float4(a.x * k, a.y * k, a.z * k, a.w * k); }
+__device__ __forceinline__ float4 f4_fma(float4 a, float k, float4 c) {
+    return make_float4(fmaf(a.x, k, c.x), fmaf(a.y, k, c.y), fmaf(a.z, k, c.z), fmaf(a.w, k, c.w));
+}
+
+template <int B>
+__device__ __forceinline__ void stage_blocks_t(float *v, int n_rg, int R4, int d, int s, const float *__restrict__ Kt, int transpose) {
+    const int nblk = d / B;
+    for (int c = threadIdx.x; c < nblk; c += blockDim.x) {
+        const int alpha = c / s, beta = c - alpha * s;
+        const int base = alpha * B * s + beta;
+        int pos[B];
+#pragma unroll
+        for (int i = 0; i < B; ++i) pos[i] = tpos(base + i * s) * R4;
+        float K[B][B];
+        const float *Kc = Kt + c;                // element-major: entry k of block c at Kt[k * nblk + c]
+#pragma unroll
+        for (int i = 0; i < B; ++i)
+#pragma unroll
+            for (int j = 0; j < B; ++j) K[i][j] = __ldg(Kc + (size_t)(transpose ? j * B + i : i * B + j) * nblk);
+#pragma unroll 2
+        for (int rg = 0; rg < n_rg; ++rg) {
+            float4 in[B];
+#pragma unroll
+            for (int i = 0; i < B; ++i) in[i] = *reinterpret_cast<const float4 *>(v + pos[i] + 4 * rg);
+#pragma unroll
+            for (int j = 0; j < B; ++j) {
+                float4 a = f4_scale(in[0], K[0][j]);
+#pragma unroll
+                for (int i = 1; i < B; ++i) a = f4_fma(in[i], K[i][j], a);
+                *reinterpret_cast<float4 *>(v + pos[j] + 4 * rg) = a;
+            }
+        }
+    }
+}
+
+template <typename T, int NT, bool BIG>
+__global__ void __launch_bounds__(NT, 1)
+harp_rowvec_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_cta, int R4, StageTable st,
+                   const float *__restrict__ blocks, const int32_t *__restrict__ perm,
+                   const int8_t *__restrict__ signs, int transpose) {
+    extern __shared__ __align__(16) float v[];       // [d][R4]
+    const int64_t row0 = (int64_t)blockIdx.x * rows_per_cta;
+    const int rows = (int)min((int64_t)rows_per_cta, n_rows - row0);
+    const int n_rg = (rows + 3) >> 2;
+    T *xt = x + row0 * d;
+    const bool aligned = d % 4 == 0 && (reinterpret_cast<uintptr_t>(x) % (4 * sizeof(T))) == 0;
+    // a1-a3: load, sign, gather (forward) -- or plain load (transpose)
+    if (aligned && (transpose || !perm)) {
+        const int nq = d >> 2;
+        for (int w = threadIdx.x; w < nq * n_rg; w += NT) {
+            const int rg = w / nq, m = w - rg * nq;
+            float e[4][4];
+#pragma unroll
+            for (int rr = 0; rr < 4; ++rr) {
+                if (4 * rg + rr < rows) load4<T>(xt + (int64_t)(4 * rg + rr) * d + 4 * m, e[rr]);
+                else e[rr][0] = e[rr][1] = e[rr][2] = e[rr][3] = 0.f;
+            }
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float sg = (!transpose && signs && signs[4 * m + k] < 0) ? -1.f : 1.f;
+                *reinterpret_cast<float4 *>(v + tpos(4 * m + k) * R4 + 4 * rg) =
+                    make_float4(sg * e[0][k], sg * e[1][k], sg * e[2][k], sg * e[3][k]);
+            }
+        }
+    } else {
+        for (int w = threadIdx.x; w < d * n_rg; w += NT) {
+            const int rg = w / d, i = w - rg * d;
+            const int src = (!transpose && perm) ? perm[i] : i;
+            const float sg = (!transpose && signs && signs[src] < 0) ? -1.f : 1.f;
+            float e[4];
+#pragma unroll
+            for (int rr = 0; rr < 4; ++rr) e[rr] = 4 * rg + rr < rows ? sg * to_f32<T>(xt[(int64_t)(4 * rg + rr) * d + src]) : 0.f;
+            *reinterpret_cast<float4 *>(v + tpos(i) * R4 + 4 * rg) = make_float4(e[0], e[1], e[2], e[3]);
+        }
+    }
+    __syncthreads();
+    for (int k = 0; k < st.m; ++k) {
+        const int t = transpose ? st.m - 1 - k : k;
+        const float *Kt = blocks + st.off[t];
+        const int b = st.b[t];
+        if (b == 2) stage_blocks_t<2>(v, n_rg, R4, d, st.s[t], Kt, transpose);
+        else if (b == 3) stage_blocks_t<3>(v, n_rg, R4, d, st.s[t], Kt, transpose);
+        else if (b == 4) stage_blocks_t<4>(v, n_rg, R4, d, st.s[t], Kt, transpose);
+        else if (BIG) {
+            if (b == 5) stage_blocks_t<5>(v, n_rg, R4, d, st.s[t], Kt, transpose);
+            else if (b == 6) stage_blocks_t<6>(v, n_rg, R4, d, st.s[t], Kt, transpose);
+            else if (b == 7) stage_blocks_t<7>(v, n_rg, R4, d, st.s[t], Kt, transpose);
+            else stage_blocks_t<8>(v, n_rg, R4, d, st.s[t], Kt, transpose);
+        }
+        __syncthreads();
+    }
+    // a5: store -- or scatter and sign (transpose)
+    if (aligned && (!transpose || !perm)) {
+        const int nq = d >> 2;
+        for (int w = threadIdx.x; w < nq * n_rg; w += NT) {
+            const int rg = w / nq, m = w - rg * nq;
+            float4 q[4];
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float sg = (transpose && signs && signs[4 * m + k] < 0) ? -1.f : 1.f;
+                q[k] = f4_scale(*reinterpret_cast<const float4 *>(v + tpos(4 * m + k) * R4 + 4 * rg), sg);
+            }
+            const float e[4][4] = {{q[0].x, q[1].x, q[2].x, q[3].x}, {q[0].y, q[1].y, q[2].y, q[3].y},
+                                   {q[0].z, q[1].z, q[2].z, q[3].z}, {q[0].w, q[1].w, q[2].w, q[3].w}};
+#pragma unroll
+            for (int rr = 0; rr < 4; ++rr)
+                if (4 * rg + rr < rows) store4<T>(xt + (int64_t)(4 * rg + rr) * d + 4 * m, e[rr]);
+        }
+    } else {
+        for (int w = threadIdx.x; w < d * n_rg; w += NT) {
+            const int rg = w / d, i = w - rg * d;
+            const int dst = (transpose && perm) ? perm[i] : i;
+            const float sg = (transpose && signs && signs[dst] < 0) ? -1.f : 1.f;
+            const float4 q = *reinterpret_cast<const float4 *>(v + tpos(i) * R4 + 4 * rg);
+            const float e[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+            for (int rr = 0; rr < 4; ++rr)
+                if (4 * rg + rr < rows) xt[(int64_t)(4 * rg + rr) * d + dst] = from_f32<T>(sg * e[rr]);
+        }
+    }
+}
+
+template <typename T, int NT, bool BIG>
+harp_status_t launch_rowvec(const harp_plan *plan, const StageTable &st, const float *blocks, void *x, int64_t n_rows,
+                            int transpose, cudaStream_t stream) {
+    auto kern = harp_rowvec_kernel<T, NT, BIG>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+        return HARP_ERR_CUDA;
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int64_t d = plan->d;
+    // groups of four rows per CTA: an odd number (bank spread), as many as shared memory holds,
+    // but no more than one wave of CTAs needs
+    int64_t g_max = (226 * 1024) / (d * 16);
+    if (g_max % 2 == 0) --g_max;
+    if (g_max < 1) return HARP_ERR_UNSUPPORTED;
+    int64_t g = ((n_rows + sms - 1) / sms + 3) / 4;
+    g = std::max<int64_t>(1, std::min<int64_t>(g, std::min<int64_t>(g_max, 15)));
+    const int64_t g_pad = g | 1;                     // g_pad <= g_max because g_max is odd
+    const int64_t r = 4 * g;
+    const int64_t grid = (n_rows + r - 1) / r;
+    if (grid > 0x7fffffffLL) return HARP_ERR_BAD_DIM;
+    kern<<<(unsigned)grid, NT, (size_t)d * 16 * g_pad, stream>>>((T *)x, n_rows, (int)d, (int)r, (int)(4 * g_pad), st, blocks,
+                                                              plan->d_perm, plan->d_signs, transpose);
+    g_harp_launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError() == cudaSuccess ? HARP_OK : HARP_ERR_CUDA;
+}
+
 template <typename T, int ITEMS>
 harp_status_t launch(const harp_plan *plan, void *x, int64_t n_rows, int rows_per_cta, int transpose,
                      cudaStream_t stream) {
@@ -330,7 +484,31 @@ harp_status_t harp_generic_build(harp_plan *plan) {
         groups.push_back({t, t1, (int)prod, plan->st.s[t], 0, 1});
         t = t1;
     }
-    if ((int)groups.size() == m) return HARP_OK;                       // nothing to fuse
+    // element-major copy of the block kernels of stage table tab (see harp_plan::d_bo_blocks)
+    auto upload_element_major = [&](const StageTable &tab, const float *src) -> harp_status_t {
+        size_t total = 0;
+        for (int t = 0; t < tab.m; ++t) total = std::max(total, (size_t)tab.off[t] + (size_t)d * tab.b[t]);
+        std::vector<float> em;
+        try {
+            em.resize(total);
+        } catch (const std::bad_alloc &) {
+            return HARP_ERR_ALLOC;
+        }
+        for (int t = 0; t < tab.m; ++t) {
+            const int b = tab.b[t];
+            const int64_t nblk = d / b;
+            for (int64_t c = 0; c < nblk; ++c)
+                for (int k = 0; k < b * b; ++k) em[(size_t)(tab.off[t] + k * nblk + c)] = src[tab.off[t] + c * b * b + k];
+        }
+        if (cudaMalloc(&plan->d_bo_blocks, sizeof(float) * std::max<size_t>(1, total)) != cudaSuccess) return HARP_ERR_ALLOC;
+        if (cudaMemcpy(plan->d_bo_blocks, em.data(), sizeof(float) * total, cudaMemcpyHostToDevice) != cudaSuccess)
+            return HARP_ERR_CUDA;
+        return HARP_OK;
+    };
+    int max_b = 0;
+    for (int t = 0; t < m; ++t) max_b = std::max(max_b, (int)plan->st.b[t]);
+    if ((int)groups.size() == m)                                        // nothing to fuse
+        return max_b <= 8 ? upload_element_major(plan->st, plan->h_blocks.data()) : HARP_OK;
     StageTable ft{};
     ft.m = (int32_t)groups.size();
     int64_t off = 0;
@@ -361,7 +539,9 @@ harp_status_t harp_generic_build(harp_plan *plan) {
     if (cudaMemcpy(plan->d_fused_blocks, fb.data(), sizeof(float) * (size_t)off, cudaMemcpyHostToDevice) != cudaSuccess)
         return HARP_ERR_CUDA;
     plan->fused = ft;
-    return HARP_OK;
+    int max_fb = 0;
+    for (int t = 0; t < ft.m; ++t) max_fb = std::max(max_fb, (int)ft.b[t]);
+    return max_fb <= 8 ? upload_element_major(ft, fb.data()) : HARP_OK;
 }
 
 harp_status_t harp_generic_supported(const harp_plan *plan, harp_dtype_t dtype) {
@@ -378,9 +558,19 @@ harp_status_t harp_generic_apply(const harp_plan *plan, void *x, int64_t n_rows,
     const int64_t d = plan->d;
     const bool use_fused = plan->fused.m > 0 && plan->d_fused_blocks;
     const StageTable &bst = use_fused ? plan->fused : plan->st;
-    const float *bblk = use_fused ? plan->d_fused_blocks : plan->d_blocks;
+    const float *bblk = plan->d_bo_blocks;       // element-major, for the block-owner kernels (radices <= 8)
     int max_radix = 0;
     for (int t = 0; t < bst.m; ++t) max_radix = std::max(max_radix, (int)bst.b[t]);
+    if (max_radix <= 8 && !bblk) return HARP_ERR_UNSUPPORTED;
+    const bool rowvec = d % 32 == 0 && d * 16 <= 226 * 1024 && !getenv("HARP_NO_ROWVEC");
+    if (rowvec && max_radix <= 4) {
+        return dtype == HARP_F32 ? launch_rowvec<float, 1024, false>(plan, bst, bblk, x, n_rows, transpose, stream)
+                                 : launch_rowvec<__nv_bfloat16, 1024, false>(plan, bst, bblk, x, n_rows, transpose, stream);
+    }
+    if (rowvec && max_radix <= 8) {
+        return dtype == HARP_F32 ? launch_rowvec<float, 256, true>(plan, bst, bblk, x, n_rows, transpose, stream)
+                                 : launch_rowvec<__nv_bfloat16, 256, true>(plan, bst, bblk, x, n_rows, transpose, stream);
+    }
     if (max_radix <= 4) {      // 1024 threads, 64 registers: the block kernel takes at most 16 of them
         return dtype == HARP_F32 ? launch_blockowner<float, 1024, false>(plan, bst, bblk, x, n_rows, transpose, stream)
                                  : launch_blockowner<__nv_bfloat16, 1024, false>(plan, bst, bblk, x, n_rows, transpose, stream);

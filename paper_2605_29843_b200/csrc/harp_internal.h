@@ -34,6 +34,10 @@ struct harp_plan {
     // stages for the CUDA-core kernel); fused.m == 0 if nothing could be fused
     StageTable fused{};
     float *d_fused_blocks = nullptr;
+    // block kernels of the stage table the block-owner kernels use (fused if present, else st),
+    // element-major: entry k = i*b + j of block c of stage t at off[t] + k * (d / b_t) + c, so that
+    // neighbouring threads (neighbouring blocks) read neighbouring words
+    float *d_bo_blocks = nullptr;
     int32_t *d_perm = nullptr;        // nullptr = identity
     int8_t *d_signs = nullptr;        // nullptr = all +1
     // host copies (used to derive kernel-specific layouts)
