@@ -67,6 +67,7 @@ stats_kernel(const T *__restrict__ A, int64_t m, int64_t n, int64_t block, doubl
         int64_t cb[V];
 #pragma unroll
         for (int v = 0; v < V; ++v) cb[v] = block > 0 ? (c0 + v) / block : -1;
+#pragma unroll 4
         for (int64_t r = blockIdx.y; r < m; r += gridDim.y) {
             const int64_t rb = block > 0 ? r / block : -2;
             float a[V];
@@ -99,6 +100,7 @@ diag_error_kernel(const T *__restrict__ Wt, const T *__restrict__ Wq, int64_t d_
             w[v] = fabs((double)to_f32<TH>(H[(c0 + v) * d_in + (c0 + v)]));
             wsum += w[v];
         }
+#pragma unroll 4
         for (int64_t r = blockIdx.y; r < d_out; r += gridDim.y) {
             float a[V], b[V];
             load_vec<T, V>(Wt + r * d_in + c0, a);

@@ -564,8 +564,8 @@ harp_status_t harp_generic_apply(const harp_plan *plan, void *x, int64_t n_rows,
     if (max_radix <= 8 && !bblk) return HARP_ERR_UNSUPPORTED;
     const bool rowvec = d % 32 == 0 && d * 16 <= 226 * 1024 && !getenv("HARP_NO_ROWVEC");
     if (rowvec && max_radix <= 4) {
-        return dtype == HARP_F32 ? launch_rowvec<float, 1024, false>(plan, bst, bblk, x, n_rows, transpose, stream)
-                                 : launch_rowvec<__nv_bfloat16, 1024, false>(plan, bst, bblk, x, n_rows, transpose, stream);
+        return dtype == HARP_F32 ? launch_rowvec<float, 512, false>(plan, bst, bblk, x, n_rows, transpose, stream)
+                                 : launch_rowvec<__nv_bfloat16, 512, false>(plan, bst, bblk, x, n_rows, transpose, stream);
     }
     if (rowvec && max_radix <= 8) {
         return dtype == HARP_F32 ? launch_rowvec<float, 256, true>(plan, bst, bblk, x, n_rows, transpose, stream)
