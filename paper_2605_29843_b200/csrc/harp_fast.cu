@@ -146,7 +146,7 @@ constexpr uint32_t kModesReorderIn2 = bit(MODE_SS) | bit(MODE_PI2);
 
 template <int NT, uint32_t MODES>
 __global__ void __launch_bounds__(NT, 1)
-harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles, FastParams P) {
+harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles, int stagger, FastParams P) {
     constexpr int NW = NT / 32;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     TileCtx c;
@@ -163,6 +163,14 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
     __syncthreads();
     const int warp = c.warp, lane = c.lane;
 
+    // All CTAs have the same work, so without this they copy their tiles in step and share the
+    // HBM bandwidth at those moments while it idles during the phases.  Three classes of CTAs
+    // start a quarter of a tile period apart (a bounded wait on the clock; only used when every
+    // CTA has several tiles, so the delay is small against the run).
+    if (stagger > 0) {
+        const long long wait = (long long)(blockIdx.x % 3) * stagger, t0 = clock64();
+        while (clock64() - t0 < wait) { }
+    }
     for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
         const int64_t row0 = tile * kTileRows;
         // rows past the end of the batch are computed on a copy of the last row and never stored
@@ -1050,11 +1058,14 @@ harp_status_t harp_fast_apply(const harp_plan *plan, void *x, int64_t n_rows, ha
     const int grid = (int)std::min<int64_t>(n_tiles, fp->max_ctas);
     __nv_bfloat16 *xb = static_cast<__nv_bfloat16 *>(x);
     const FastParams &P = transpose ? fp->bwd : fp->fwd;
+    // a quarter of a tile period, estimated from the measured 28 k cycles per tile of d = 4096 with
+    // three phases (the gain is flat between half and the full value)
+    const int stagger = n_tiles >= 4 * (int64_t)grid ? (int)(0.57 * (double)P.d * P.n_phases) : 0;
     switch (transpose ? fp->variant_bwd : fp->variant_fwd) {
-        case 1: harp_fast_kernel<kThreads, kModesReorderOut><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, P); break;
-        case 2: harp_fast_kernel<kThreads, kModesReorderIn><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, P); break;
-        case 3: harp_fast_kernel<kThreads, kModesReorderIn2><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, P); break;
-        default: harp_fast_kernel<kThreads, kModesGeneral><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, P); break;
+        case 1: harp_fast_kernel<kThreads, kModesReorderOut><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, stagger, P); break;
+        case 2: harp_fast_kernel<kThreads, kModesReorderIn><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, stagger, P); break;
+        case 3: harp_fast_kernel<kThreads, kModesReorderIn2><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, stagger, P); break;
+        default: harp_fast_kernel<kThreads, kModesGeneral><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, stagger, P); break;
     }
     g_harp_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HARP_OK : HARP_ERR_CUDA;
