@@ -18,15 +18,13 @@
 //
 // Permutations.  Identity: the tile is copied in and out with coalesced 16-byte accesses.
 // Mixed-radix digit reversal of the plan's own schedule: the tile is copied in coalesced in
-// source order, the phases run in place on the source-ordered layout (a digit reversal
-// maps every phase onto a digit group again, only with other strides), and the one phase
-// next to the output does the reordering inside shared memory.  Forward: an item of that
-// phase reads eight blocks that are neighbours in output order (16 contiguous source values
-// each, ldmatrix) and writes its sixteen eight-block runs into the same sixteen 16-byte
-// slots, so the phase is in place and the copy to global memory follows a chunk map.
-// Transpose: all operands of the phase are read from an output-ordered layout into registers,
-// the CTA synchronises, and the results are written as contiguous source blocks (the in-place
-// form of this direction exists too, but measures slower).
+// the order of the direction's input (source order forward, output order for the transpose),
+// the phases run in place on a layout ordered the same way (a digit reversal maps every phase
+// onto a digit group again, only with other strides), and the last phase of the direction
+// reorders inside shared memory, in place: an item of that phase reads eight blocks that are
+// neighbours in the order of the direction's output (16 contiguous values of the layout each,
+// ldmatrix) and writes its sixteen eight-block runs into the same sixteen 16-byte slots; the
+// copy to global memory follows a chunk map.
 // Any other permutation that maps every aligned run of eight source coordinates onto the
 // same slot of eight different first-phase blocks is gathered (forward) or scattered
 // (transpose) in global memory with 16-byte accesses by the first/last phase.  All other
@@ -54,9 +52,7 @@ enum PhaseMode : int32_t {
     MODE_SS = 1,   // strided block in shared memory, eight blocks per item, in place
     MODE_GS = 2,   // operands gathered from global memory, result to contiguous smem blocks
     MODE_CG = 3,   // operands from contiguous smem blocks, result scattered to global memory
-    MODE_PO = 4,   // contiguous smem blocks in, eight-block runs out to the same slots (reorders the tile in place)
-    MODE_PI = 5,   // strided smem in (output-ordered layout), CTA barrier, contiguous smem blocks out
-    MODE_PI2 = 6   // eight-block runs in, contiguous smem blocks out to the same slots (in place)
+    MODE_PO = 4    // contiguous smem blocks in, eight-block runs out to the same slots (reorders the tile in place)
 };
 
 struct PhaseDesc {
@@ -140,9 +136,7 @@ __device__ __forceinline__ void gs_store(const TileCtx &c, const PhaseDesc &ph, 
 // scheme does not pay for the others.
 __host__ __device__ constexpr uint32_t bit(int mode) { return 1u << mode; }
 constexpr uint32_t kModesGeneral = bit(MODE_CC) | bit(MODE_SS) | bit(MODE_GS) | bit(MODE_CG);
-constexpr uint32_t kModesReorderOut = bit(MODE_SS) | bit(MODE_PO);
-constexpr uint32_t kModesReorderIn = bit(MODE_SS) | bit(MODE_PI);
-constexpr uint32_t kModesReorderIn2 = bit(MODE_SS) | bit(MODE_PI2);
+constexpr uint32_t kModesReorderOut = bit(MODE_SS) | bit(MODE_PO);   // the digit-reversal scheme, both directions
 
 template <int NT, uint32_t MODES>
 __global__ void __launch_bounds__(NT, 1)
@@ -337,72 +331,6 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
                         sts128(o0 + 2u * (uint32_t)(8 * pitch), out[j][1]);
                     }
                 }
-            } else if ((MODES & bit(MODE_PI)) && ph.mode == MODE_PI) {
-                const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
-                const int it0 = warp, it1 = warp + NW;
-                uint32_t mats[8][4];
-                uint4 raw1[4][2];
-                if (it0 < n) {
-                    const uint32_t i0 = c.sbase + 2u * (uint32_t)(c.g * pitch + c.q * ph.lane_step + tab_s[ph.items_off + it0 * 12 + 8]);
-                    const uint32_t i1 = i0 + 2u * (uint32_t)(8 * pitch);
-                    uint4 raw[4][2], bf[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) bf[e] = __ldg(ph.bfrag + (size_t)it0 * 256 + e * 32 + lane);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        raw[j][0] = lds128(i0 + 2u * ph.j_off[j]);
-                        raw[j][1] = lds128(i1 + 2u * ph.j_off[j]);
-                    }
-                    octet_mma16<false>(raw, bf, mats);
-                }
-                if (it1 < n) {
-                    const uint32_t i0 = c.sbase + 2u * (uint32_t)(c.g * pitch + c.q * ph.lane_step + tab_s[ph.items_off + it1 * 12 + 8]);
-                    const uint32_t i1 = i0 + 2u * (uint32_t)(8 * pitch);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        raw1[j][0] = lds128(i0 + 2u * ph.j_off[j]);
-                        raw1[j][1] = lds128(i1 + 2u * ph.j_off[j]);
-                    }
-                }
-                __syncthreads();
-                if (it0 < n) {
-                    const int32_t *tab = tab_s + ph.items_off + it0 * 12;
-#pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        stmatrix_x4(c.sbase + 2u * (uint32_t)(mrow * pitch + tab[e] + mcol), mats[e][0], mats[e][1], mats[e][2], mats[e][3]);
-                }
-                if (it1 < n) {
-                    uint4 bf[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) bf[e] = __ldg(ph.bfrag + (size_t)it1 * 256 + e * 32 + lane);
-                    octet_mma16<false>(raw1, bf, mats);
-                    const int32_t *tab = tab_s + ph.items_off + it1 * 12;
-#pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        stmatrix_x4(c.sbase + 2u * (uint32_t)(mrow * pitch + tab[e] + mcol), mats[e][0], mats[e][1], mats[e][2], mats[e][3]);
-                }
-            } else if ((MODES & bit(MODE_PI2)) && ph.mode == MODE_PI2) {
-                // the reverse: sixteen slots in (eight-block runs), contiguous blocks out (stmatrix)
-                // to the same slots
-                const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
-                for (int it = warp; it < n; it += NW) {
-                    const int32_t *tab = tab_s + ph.items_off + it * 24;
-                    uint4 raw[4][2], bf[8];
-                    uint32_t mats[8][4];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) bf[e] = __ldg(ph.bfrag + (size_t)it * 256 + e * 32 + lane);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const uint32_t i0 = c.sbase + 2u * (uint32_t)(c.g * pitch + tab[8 + c.q + 4 * j]);
-                        raw[j][0] = lds128(i0);
-                        raw[j][1] = lds128(i0 + 2u * (uint32_t)(8 * pitch));
-                    }
-                    octet_mma16<false>(raw, bf, mats);
-                    __syncwarp();
-#pragma unroll
-                    for (int e = 0; e < 8; ++e)
-                        stmatrix_x4(c.sbase + 2u * (uint32_t)(mrow * pitch + tab[e] + mcol), mats[e][0], mats[e][1], mats[e][2], mats[e][3]);
-                }
             } else if ((MODES & bit(MODE_CG)) && ph.mode == MODE_CG) {   // operands from contiguous smem blocks, results scattered to global memory
                 const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
                 for (int it = warp; it < n; it += NW) {
@@ -595,17 +523,23 @@ harp_status_t harp_fast_build(harp_plan *plan) {
         for (int p = 0; p < np; ++p) o += L.off(p, (pos / L.S[(size_t)p]) % phases[(size_t)p].B);
         return o;
     };
-    // In the digit-reversal scheme the output-ordered chunk map follows from the source layout:
-    // chunk (hi + lo + r*S)/8 of the output lives in slot (e, h) = (r & 7, r >> 3) of the item's
-    // eight source blocks (see reorder_slots below).
-    auto reorder_off = [&](const Layout &L, int64_t hi, int64_t lo, int sl) {
-        return phys_in(L, plan->h_perm[(size_t)(hi + lo + (sl & 7))]) + 8 * (sl >> 3);
+    // In the digit-reversal scheme the phases run on the layout ordered like the input of the
+    // direction (source order forward, output order for the transpose) and the last phase reorders
+    // in place: an item is eight blocks that are neighbours in the direction's output order
+    // (coordinates hi + lo + e there), each 16 contiguous coordinates of the layout, and slot
+    // (e, h) = (sl & 7, sl >> 3) of these sixteen 16-byte slots receives one run of eight
+    // neighbouring output coordinates (see reorder_slots below).
+    auto reorder_off = [&](const Layout &L, int dir, int64_t hi, int64_t lo, int sl) {
+        const int64_t co = hi + lo + (sl & 7);
+        return phys_in(L, dir == 0 ? (int64_t)plan->h_perm[(size_t)co] : inv[(size_t)co]) + 8 * (sl >> 3);
     };
-    auto layout_cost = [&](const Layout &L, bool src_scheme) {
+    // scheme 0: plain (both tile copies follow the layout); 1: L is the source-ordered layout of
+    // the forward reordering scheme; 2: L is the output-ordered layout of the transpose one
+    auto layout_cost = [&](const Layout &L, int scheme) {
         const int64_t pc = pitch_of(L) / 8;
         double cost = 1e-7 * (double)L.extent;
         // strided phases: lanes q = 0..3 of two neighbouring rows
-        const std::vector<int> &order = src_scheme ? order_src : order_nat;
+        const std::vector<int> &order = scheme == 1 ? order_src : order_nat;
         for (size_t k = 1; k < order.size(); ++k) {
             const int p = order[k];
             const int64_t step = L.lm[(size_t)p] * L.W[(size_t)p] + (L.lm[(size_t)p] == 4 ? L.gp[(size_t)p] : 0);
@@ -625,18 +559,20 @@ harp_status_t harp_fast_build(harp_plan *plan) {
             return sum / (double)((d / 8 + 7) / 8);
         };
         cost += map_cost([&](int64_t c) { return phys_in(L, 8 * c); });
-        if (src_scheme) {
-            const HostPhase &hp = phases[(size_t)np - 1];
+        if (scheme != 0) {
+            // stride of the reordering phase in the order of the direction's output
+            const int pr = scheme == 1 ? np - 1 : 0;
+            const int64_t So = scheme == 1 ? phases[(size_t)pr].S : S_src[(size_t)pr], Bo = phases[(size_t)pr].B;
             cost += map_cost([&](int64_t c) {
-                const int64_t o = 8 * c, span = hp.S * hp.B;                         // o = hi + lo + r*S
-                return reorder_off(L, o / span * span, o % hp.S, (int)((o / hp.S) % hp.B));
+                const int64_t o = 8 * c, span = So * Bo;                              // o = hi + lo + r*So
+                return reorder_off(L, scheme - 1, o / span * span, o % So, (int)((o / So) % Bo));
             });
         } else {
             cost += map_cost([&](int64_t c) { return phys_in(L, 8 * c); });
         }
         return cost;
     };
-    auto search_layout = [&](const std::vector<int> &order, const std::vector<int64_t> &strides, bool src_scheme, Layout &best) {
+    auto search_layout = [&](const std::vector<int> &order, const std::vector<int64_t> &strides, int src_scheme, Layout &best) {
         // start: the smallest padding that makes every strided phase conflict-free on its own
         std::vector<Choice> ch((size_t)np, Choice{0, 0, 1});
         {
@@ -704,9 +640,9 @@ harp_status_t harp_fast_build(harp_plan *plan) {
         return true;
     };
     Layout Lnat, Lsrc;
-    if (!search_layout(order_nat, S_nat, false, Lnat)) return HARP_ERR_UNSUPPORTED;
+    if (!search_layout(order_nat, S_nat, digitrev ? 2 : 0, Lnat)) return HARP_ERR_UNSUPPORTED;
     if (digitrev) {
-        if (!search_layout(order_src, S_src, true, Lsrc)) return HARP_ERR_UNSUPPORTED;
+        if (!search_layout(order_src, S_src, 1, Lsrc)) return HARP_ERR_UNSUPPORTED;
     } else {
         Lsrc = Lnat;
     }
@@ -763,17 +699,16 @@ harp_status_t harp_fast_build(harp_plan *plan) {
         chunk_nat[(size_t)c] = (int32_t)phys_nat(8 * c);
         chunk_src[(size_t)c] = (int32_t)phys_src(8 * c);
     }
-    const std::vector<int32_t> chunk_nat_plain(chunk_nat);   // output order in the output-ordered layout
-    // Digit reversal: the phase next to the output reorders the tile in place.  An item is eight
-    // blocks that are neighbours in output order; each is 16 contiguous source coordinates, so the
-    // item owns sixteen 16-byte slots of the source-ordered layout.  After the phase slot
-    // (e, h) = (s & 7, s >> 3), s = slot_of[r], holds, for output local index r, the eight blocks'
-    // values: a run of eight neighbouring output coordinates.  reorder_slots[item][r] is that
-    // slot's offset, and the output-ordered chunk map follows from it.
-    std::vector<int32_t> reorder_slots;
-    if (digitrev) {
-        const HostPhase &hp = phases[(size_t)np - 1];
-        const int64_t span = hp.S * hp.B;
+    // Digit reversal: the last phase of either direction reorders the tile in place (see
+    // reorder_off).  After it slot slot_of[r] of an item holds, for local index r in output order,
+    // the eight blocks' values: a run of eight neighbouring output coordinates.
+    // reorder_slots[dir][item][r] is that slot's offset and chunk_out[dir] the chunk map of the
+    // copy to global memory that follows from it.
+    std::vector<int32_t> reorder_slots[2], chunk_out[2];
+    for (int dir = 0; dir < 2 && digitrev; ++dir) {
+        const Layout &L = dir == 0 ? Lsrc : Lnat;
+        const int pr = dir == 0 ? np - 1 : 0;
+        const int64_t So = dir == 0 ? phases[(size_t)pr].S : S_src[(size_t)pr], span = So * phases[(size_t)pr].B;
         // The four lanes q of a quarter-warp access the slots of r = q + 4j in two neighbouring
         // rows.  Starting from the identity, swap pairs while that lowers the number of
         // shared-memory wavefronts (judged on the first item; the other items differ by a
@@ -785,7 +720,7 @@ harp_status_t harp_fast_build(harp_plan *plan) {
             for (int j = 0; j < 4; ++j) {
                 std::vector<int64_t> slots;
                 for (int q = 0; q < 4; ++q)
-                    for (int row = 0; row < 2; ++row) slots.push_back(reorder_off(Lsrc, 0, 0, slot_of[q + 4 * j]) / 8 + row * (pitch / 8));
+                    for (int row = 0; row < 2; ++row) slots.push_back(reorder_off(L, dir, 0, 0, slot_of[q + 4 * j]) / 8 + row * (pitch / 8));
                 total += worst_bank(slots);
             }
             return total;
@@ -800,18 +735,15 @@ harp_status_t harp_fast_build(harp_plan *plan) {
                     else std::swap(slot_of[a], slot_of[b]);
                 }
         }
+        chunk_out[dir].assign((size_t)(d / 8), 0);
         for (int64_t hi = 0; hi < d; hi += span)
-            for (int64_t lo = 0; lo < hp.S; lo += 8)
+            for (int64_t lo = 0; lo < So; lo += 8)
                 for (int r = 0; r < 16; ++r) {
-                    const int32_t off = (int32_t)reorder_off(Lsrc, hi, lo, slot_of[r]);
-                    reorder_slots.push_back(off);
-                    chunk_nat[(size_t)((hi + lo + (int64_t)r * hp.S) / 8)] = off;
+                    const int32_t off = (int32_t)reorder_off(L, dir, hi, lo, slot_of[r]);
+                    reorder_slots[dir].push_back(off);
+                    chunk_out[dir][(size_t)((hi + lo + (int64_t)r * So) / 8)] = off;
                 }
     }
-
-    // digit reversal, transpose direction: the barrier variant of the reordering phase (a warp
-    // holds at most two items over the barrier) measures faster than the in-place one
-    const bool pi_barrier = digitrev && d / 16 / 8 <= 2 * (kThreads / 32);
 
     auto sign_v = [&](int64_t i) -> double {             // sign seen by coordinate i after the gather
         if (plan->h_signs.empty()) return 1.0;
@@ -826,20 +758,20 @@ harp_status_t harp_fast_build(harp_plan *plan) {
         P.n_phases = np;
         P.d = (int32_t)d;
         P.pitch = (int32_t)pitch;
-        // chunk maps: output order (for the digit-reversal scheme: where the in-place reordering
-        // phase leaves / expects it), source order, and output order in the output-ordered layout
+        // chunk maps: output order and source order in their layouts, and (digit reversal) where the
+        // in-place reordering phase of this direction leaves the chunks of its output
         std::vector<int32_t> tables(chunk_nat);
         const int32_t off_nat = 0;
         const int32_t off_src = (int32_t)tables.size();
         tables.insert(tables.end(), chunk_src.begin(), chunk_src.end());
-        const int32_t off_natl = (int32_t)tables.size();
-        if (digitrev && pi_barrier) tables.insert(tables.end(), chunk_nat_plain.begin(), chunk_nat_plain.end());
+        const int32_t off_out = (int32_t)tables.size();
+        if (digitrev) tables.insert(tables.end(), chunk_out[dir].begin(), chunk_out[dir].end());
         if (identity) {
             P.copy_in = off_nat;
             P.copy_out = off_nat;
         } else if (digitrev) {
-            P.copy_in = dir == 0 ? off_src : (pi_barrier ? off_natl : off_nat);
-            P.copy_out = dir == 0 ? off_nat : off_src;
+            P.copy_in = dir == 0 ? off_src : off_nat;
+            P.copy_out = off_out;
         } else {
             P.copy_in = dir == 0 ? -1 : off_nat;
             P.copy_out = dir == 0 ? off_nat : -1;
@@ -851,14 +783,16 @@ harp_status_t harp_fast_build(harp_plan *plan) {
             const int B = hp.B;
             int mode;
             if (identity) mode = p == 0 ? MODE_CC : MODE_SS;
-            else if (digitrev) mode = p == np - 1 ? (dir == 0 ? MODE_PO : (pi_barrier ? MODE_PI : MODE_PI2)) : MODE_SS;
+            else if (digitrev) mode = p == (dir == 0 ? np - 1 : 0) ? MODE_PO : MODE_SS;
             else mode = p == 0 ? (dir == 0 ? MODE_GS : MODE_CG) : MODE_SS;
             D.mode = mode;
             D.B = B;
             // Which layout do the strided accesses of this phase use, and with which slot geometry?
-            const bool src_side = digitrev && mode == MODE_SS;          // in place on the source-ordered layout
+            // digit reversal: the forward direction works on the source-ordered layout, the transpose
+            // on the output-ordered one
+            const bool src_side = digitrev && dir == 0 && mode == MODE_SS;
             const Layout &L = src_side ? Lsrc : Lnat;
-            const int lm = (mode == MODE_GS || mode == MODE_CG || mode == MODE_CC || mode == MODE_PO || mode == MODE_PI2)
+            const int lm = (mode == MODE_GS || mode == MODE_CG || mode == MODE_CC || mode == MODE_PO)
                                ? 1 : L.lm[(size_t)p];   // table-indexed slots use the plain map
             const int *jo = B == 16 ? (lm == 1 ? joff1_16 : lm == 2 ? joff2_16 : joff4_16) : (lm == 1 ? joff1_8 : joff2_8);
             if (mode == MODE_GS || mode == MODE_CG) {    // these index the item table by slot
@@ -872,10 +806,13 @@ harp_status_t harp_fast_build(harp_plan *plan) {
             // local index seen by the strided / contiguous side of the operand, as a natural local index
             auto strided_nat = [&](int slot) {
                 const int r = strided_slot(slot, B, lm);
-                return src_side ? nat_local_of_src_local(p, r) : r;
+                // the strided side counts in source order in the forward in-place phases and in the
+                // reordering phase of the transpose, whose output is source-ordered
+                const bool in_src_order = src_side || (mode == MODE_PO && dir == 1);
+                return in_src_order ? nat_local_of_src_local(p, r) : r;
             };
-            auto contig_nat = [&](int slot) {            // contiguous blocks of PO/PI live in the source layout
-                return (mode == MODE_PO || mode == MODE_PI || mode == MODE_PI2) ? nat_local_of_src_local(p, slot) : slot;
+            auto contig_nat = [&](int slot) {            // the forward reordering phase reads contiguous source blocks
+                return (mode == MODE_PO && dir == 0) ? nat_local_of_src_local(p, slot) : slot;
             };
             // enumerate items and the natural base coordinate of every block
             std::vector<int32_t> items;
@@ -901,32 +838,21 @@ harp_status_t harp_fast_build(harp_plan *plan) {
                         items.push_back((int32_t)phys_src(hi + lo));
                         for (int e = 0; e < 8; ++e) block_base.push_back(inv[(size_t)(hi + lo + e)]);
                     }
-            } else if (mode == MODE_PI) {
-                // as below, but the strided side lives in the output-ordered layout
-                ints_per_item = 12;
-                const int64_t span = hp.S * B;
-                for (int64_t hi = 0; hi < d; hi += span)
-                    for (int64_t lo = 0; lo < hp.S; lo += 8) {
-                        for (int e = 0; e < 8; ++e) {
-                            items.push_back((int32_t)phys_src(plan->h_perm[(size_t)(hi + lo + e)]));
-                            block_base.push_back(hi + lo + e);
-                        }
-                        items.push_back((int32_t)phys_nat(hi + lo));
-                        items.push_back(0); items.push_back(0); items.push_back(0);
-                    }
-            } else if (mode == MODE_PO || mode == MODE_PI2) {
-                // octets of blocks that are neighbours in natural order; each block is 16 contiguous
-                // source coordinates
+            } else if (mode == MODE_PO) {
+                // octets of blocks that are neighbours in the order of this direction's output; each
+                // block is 16 contiguous coordinates of the layout the direction works on
                 ints_per_item = 24;
-                const int64_t span = hp.S * B;
+                const int64_t So = dir == 0 ? hp.S : S_src[(size_t)p], span = So * B;
                 size_t item_no = 0;
                 for (int64_t hi = 0; hi < d; hi += span)
-                    for (int64_t lo = 0; lo < hp.S; lo += 8, ++item_no) {
+                    for (int64_t lo = 0; lo < So; lo += 8, ++item_no) {
                         for (int e = 0; e < 8; ++e) {
-                            items.push_back((int32_t)phys_src(plan->h_perm[(size_t)(hi + lo + e)]));
-                            block_base.push_back(hi + lo + e);
+                            // natural coordinate of the block's local index 0
+                            const int64_t nb = dir == 0 ? hi + lo + e : inv[(size_t)(hi + lo + e)];
+                            items.push_back((int32_t)(dir == 0 ? phys_src(plan->h_perm[(size_t)nb]) : phys_nat(nb)));
+                            block_base.push_back(nb);
                         }
-                        for (int r = 0; r < 16; ++r) items.push_back(reorder_slots[item_no * 16 + (size_t)r]);
+                        for (int r = 0; r < 16; ++r) items.push_back(reorder_slots[dir][item_no * 16 + (size_t)r]);
                     }
             } else {
                 ints_per_item = 24;
@@ -957,14 +883,8 @@ harp_status_t harp_fast_build(harp_plan *plan) {
                     for (int32_t b : items) ok = ok && contig_ok(b);
                 } else if (mode == MODE_SS) {
                     for (int32_t b : items) ok = ok && strided_ok(b);
-                } else if (mode == MODE_PI) {
-                    ok = ok && B == 16 && D.n_items <= 2 * (kThreads / 32);
-                    for (size_t i = 0; i < items.size(); i += 12) {
-                        for (int e = 0; e < 8; ++e) ok = ok && contig_ok(items[i + e]);
-                        ok = ok && strided_ok(items[i + 8]);
-                    }
-                } else if (mode == MODE_PO || mode == MODE_PI2) {
-                    ok = ok && B == 16 && hp.S % 8 == 0;
+                } else if (mode == MODE_PO) {
+                    ok = ok && B == 16 && (dir == 0 ? hp.S : S_src[(size_t)p]) % 8 == 0;
                     for (size_t i = 0; i < items.size(); i += 24) {
                         for (int e = 0; e < 8; ++e) ok = ok && contig_ok(items[i + e]);
                         for (int r = 0; r < 16; ++r) ok = ok && items[i + 8 + r] >= 0 && items[i + 8 + r] % 8 == 0 && items[i + 8 + r] + 8 <= pitch;
@@ -980,7 +900,7 @@ harp_status_t harp_fast_build(harp_plan *plan) {
             D.items_off = (int32_t)tables.size();
             tables.insert(tables.end(), items.begin(), items.end());
             // fragments: B[k-slot][n-slot] = G[local index of the k-slot][local index of the n-slot]
-            const bool in_strided = (mode == MODE_SS || mode == MODE_GS || mode == MODE_PI || mode == MODE_PI2);
+            const bool in_strided = (mode == MODE_SS || mode == MODE_GS);
             const bool out_strided = (mode == MODE_SS || mode == MODE_CG || mode == MODE_PO);
             const int words_per_lane = B == 16 ? 4 : 1;
             std::vector<uint32_t> frag(block_base.size() * 32 * words_per_lane);
@@ -1022,12 +942,10 @@ harp_status_t harp_fast_build(harp_plan *plan) {
     if (st == HARP_OK && fp->smem_bytes > 227u * 1024u) st = HARP_ERR_UNSUPPORTED;
     if (st == HARP_OK) {
         if (cudaFuncSetAttribute(harp_fast_kernel<kThreads, kModesGeneral>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-            cudaFuncSetAttribute(harp_fast_kernel<kThreads, kModesReorderOut>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-            cudaFuncSetAttribute(harp_fast_kernel<kThreads, kModesReorderIn>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-            cudaFuncSetAttribute(harp_fast_kernel<kThreads, kModesReorderIn2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+            cudaFuncSetAttribute(harp_fast_kernel<kThreads, kModesReorderOut>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
             st = HARP_ERR_CUDA;
         fp->variant_fwd = digitrev ? 1 : 0;
-        fp->variant_bwd = digitrev ? (pi_barrier ? 2 : 3) : 0;
+        fp->variant_bwd = digitrev ? 1 : 0;
         int dev = 0, sms = 0;
         cudaGetDevice(&dev);
         cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -1063,8 +981,6 @@ harp_status_t harp_fast_apply(const harp_plan *plan, void *x, int64_t n_rows, ha
     const int stagger = n_tiles >= 4 * (int64_t)grid ? (int)(0.57 * (double)P.d * P.n_phases) : 0;
     switch (transpose ? fp->variant_bwd : fp->variant_fwd) {
         case 1: harp_fast_kernel<kThreads, kModesReorderOut><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, stagger, P); break;
-        case 2: harp_fast_kernel<kThreads, kModesReorderIn><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, stagger, P); break;
-        case 3: harp_fast_kernel<kThreads, kModesReorderIn2><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, stagger, P); break;
         default: harp_fast_kernel<kThreads, kModesGeneral><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, stagger, P); break;
     }
     g_harp_launches.fetch_add(1, std::memory_order_relaxed);
