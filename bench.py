@@ -35,8 +35,8 @@ WORKLOAD = "cfg2: d=4096 radix-4 x6, signs + digit-reversal perm, 16384 rows bf1
 N_BUF = 4
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of harp_fast_kernel on the
 # headline workload, mean of the forward and the transpose launch in profiles/harp_fast_kernel_cfg2.md
-# (read 134.6 / 134.7 MB, write 75.7 / 83.8 MB: the last tiles' write-back is still in L2 at kernel end).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 214_440_000
+# (read 134.6 / 134.6 MB, write 75.1 / 75.3 MB: the last tiles' write-back is still in L2 at kernel end).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 209_830_000
 
 
 def measured_peaks():
