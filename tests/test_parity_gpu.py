@@ -83,6 +83,23 @@ def test_configs_reduced_rows_all_elements(cfg, kernel):
     assert orc.rel_err_rows(back, x64) <= 2 * w.tol
 
 
+@pytest.mark.parametrize("cfg", [1, 2])
+def test_row_major_cuda_core_kernel(cfg, monkeypatch):
+    """The CUDA-core path has two tile layouts; the row-major one (used when d is not a multiple of
+    32) is forced here on dimensions that would take the transposed one, which also exercises its
+    bank swizzle (d a multiple of 128) and the 16-byte tile copies."""
+    monkeypatch.setenv("HARP_NO_ROWVEC", "1")
+    n = 37
+    w, spec, data = _cfg_plan_and_data(cfg, n)
+    plan = harp.plan_from_spec(spec)
+    cplan = c_oracle.CPlan(spec)
+    xh, x64 = data.rows(0, n), data.rows_f64(0, n)
+    got, guards = gpu_apply(plan, xh, data.dtype, False, harp.KERNEL_GENERIC)
+    assert guards and orc.rel_err_rows(got, c_oracle.forward(cplan, x64)) <= w.tol
+    got, guards = gpu_apply(plan, xh, data.dtype, True, harp.KERNEL_GENERIC)
+    assert guards and orc.rel_err_rows(got, c_oracle.transpose(cplan, x64)) <= w.tol
+
+
 @pytest.mark.parametrize("cfg", [4])
 def test_decode_batches(cfg):
     w, spec, data = _cfg_plan_and_data(cfg, 16)
