@@ -144,6 +144,18 @@ harp_status_t harp_apply_ex(const harp_plan_t *plan, void *x, int64_t n_rows,
                             harp_dtype_t dtype, int transpose, harp_kernel_t kernel,
                             void *stream);
 
+/* Several passes (Section "HARP processors": independent copies of a schedule may be composed;
+ * one pass is the paper's default).  Forward computes x <- x Q_0 Q_1 ... Q_{n-1} with
+ * Q_k = the processor of plans[k], one harp_apply per pass in that order; transpose != 0 computes
+ * x <- x Q_{n-1}^T ... Q_0^T, the inverse for orthogonal blocks.
+ *   plans     HOST array of n_passes plan handles of the same dimension (each may have its own
+ *             schedule, permutation and signs; a pass after the first usually has neither)
+ *   x         DEVICE n_rows x d, overwritten
+ * Errors: HARP_ERR_NULL, HARP_ERR_BAD_SCHEDULE (n_passes < 1), HARP_ERR_DIM_MISMATCH, and those
+ * of harp_apply (a failing pass leaves x partly transformed).  Asynchronous on stream. */
+harp_status_t harp_apply_passes(const harp_plan_t *const *plans, int32_t n_passes, void *x,
+                                int64_t n_rows, harp_dtype_t dtype, int transpose, void *stream);
+
 /* Two-sided processing of a weight matrix, W <- Q_out^T W Q_in (paper, Section
  * "Incoherence processing": W~ = U^T W V with U = Q_out, V = Q_in; Algorithm 3 line 3).
  *   W        DEVICE d_out x d_in row-major, d_out = dim(plan_out), d_in = dim(plan_in)

@@ -122,6 +122,22 @@ def two_sided(plan_out: OraclePlan, plan_in: OraclePlan, w: np.ndarray) -> np.nd
     return forward(plan_out, rows_done.T).T                     # each column . Q_out
 
 
+def forward_passes(plans: Sequence[OraclePlan], x: np.ndarray) -> np.ndarray:
+    """Several passes (Section "HARP processors"): y = x . Q_0 . Q_1 ... , each Q_k one processor."""
+    y = np.array(x, dtype=np.float64, ndmin=2)
+    for p in plans:
+        y = forward(p, y)
+    return y
+
+
+def transpose_passes(plans: Sequence[OraclePlan], y: np.ndarray) -> np.ndarray:
+    """x = y . Q_{n-1}^T ... Q_0^T, the inverse of forward_passes for orthogonal blocks."""
+    x = np.array(y, dtype=np.float64, ndmin=2)
+    for p in reversed(list(plans)):
+        x = transpose(p, x)
+    return x
+
+
 def dense(plan: OraclePlan) -> np.ndarray:
     """Materialise Q (d x d) with forward(x) == x @ Q, by pushing the identity through."""
     return forward(plan, np.eye(plan.d))

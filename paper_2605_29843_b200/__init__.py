@@ -57,6 +57,8 @@ def lib() -> ctypes.CDLL:
         L.harp_apply.argtypes = [vp, vp, i64, ctypes.c_int, ctypes.c_int, vp]
         L.harp_apply_ex.restype = ctypes.c_int
         L.harp_apply_ex.argtypes = [vp, vp, i64, ctypes.c_int, ctypes.c_int, ctypes.c_int, vp]
+        L.harp_apply_passes.restype = ctypes.c_int
+        L.harp_apply_passes.argtypes = [ctypes.POINTER(vp), i32, vp, i64, ctypes.c_int, ctypes.c_int, vp]
         L.harp_apply_two_sided.restype = ctypes.c_int
         L.harp_apply_two_sided.argtypes = [vp, ctypes.c_int, vp, vp, vp, vp]
         L.harp_two_sided_scratch_bytes.restype = i64
@@ -214,6 +216,14 @@ def harp_apply(plan: Plan, x_ptr: int, n_rows: int, dtype: int, transpose: bool 
                              int(kernel), stream or None)
     if st != HARP_OK:
         raise HarpError(st, "harp_apply")
+
+
+def harp_apply_passes(plans, x_ptr: int, n_rows: int, dtype: int, transpose: bool = False, stream: int = 0) -> None:
+    """Several passes: x <- x Q_0 Q_1 ... (or the transposes in the opposite order)."""
+    arr = (ctypes.c_void_p * len(plans))(*[p.handle for p in plans])
+    st = lib().harp_apply_passes(arr, len(plans), x_ptr, int(n_rows), int(dtype), 1 if transpose else 0, stream or None)
+    if st != HARP_OK:
+        raise HarpError(st, "harp_apply_passes")
 
 
 def harp_apply_two_sided(w_ptr: int, dtype: int, plan_out: Plan, plan_in: Plan,

@@ -192,6 +192,24 @@ extern "C" harp_status_t harp_apply(const harp_plan_t *plan, void *x, int64_t n_
     return harp_apply_ex(plan, x, n_rows, dtype, transpose, HARP_KERNEL_AUTO, stream);
 }
 
+// Several passes: forward applies plans[0], plans[1], ... in turn; the transpose undoes them in
+// the opposite order.
+extern "C" harp_status_t harp_apply_passes(const harp_plan_t *const *plans, int32_t n_passes, void *x, int64_t n_rows,
+                                           harp_dtype_t dtype, int transpose, void *stream) {
+    if (!plans) return HARP_ERR_NULL;
+    if (n_passes < 1) return HARP_ERR_BAD_SCHEDULE;
+    for (int32_t k = 0; k < n_passes; ++k) {
+        if (!plans[k]) return HARP_ERR_NULL;
+        if (plans[k]->d != plans[0]->d) return HARP_ERR_DIM_MISMATCH;
+    }
+    for (int32_t k = 0; k < n_passes; ++k) {
+        const harp_plan_t *p = plans[transpose ? n_passes - 1 - k : k];
+        const harp_status_t st = harp_apply(p, x, n_rows, dtype, transpose, stream);
+        if (st != HARP_OK) return st;
+    }
+    return HARP_OK;
+}
+
 extern "C" int64_t harp_two_sided_scratch_bytes(const harp_plan_t *plan_out, const harp_plan_t *plan_in,
                                                 harp_dtype_t dtype) {
     if (!plan_out || !plan_in || (dtype != HARP_F32 && dtype != HARP_BF16)) return 0;

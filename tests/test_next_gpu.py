@@ -86,3 +86,26 @@ def test_symmetric_two_sided_product(dtype):
     assert np.max(np.abs(got - want) / scale) <= 2 * TOL[dtype]
     assert abs(np.trace(got) - np.trace(h64)) / np.trace(h64) < (1e-5 if dtype == "f32" else 5e-3)
     assert np.max(np.abs(got - got.T) / scale) <= 4 * TOL[dtype]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_passes(dtype):
+    """Two and three passes against the oracle's composition, forward and transpose."""
+    specs = [wl.tiny_plan(11, (4, 4, 4, 4), kind="qr", perm="random", signs=True),
+             wl.tiny_plan(12, (16, 16), kind="qr", perm="identity", signs=False),
+             wl.tiny_plan(13, (2, 8, 16), kind="qr", perm="identity", signs=True)]
+    plans = [harp.plan_from_spec(sp) for sp in specs]
+    oplans = [orc.OraclePlan.from_spec(sp) for sp in specs]
+    rng = np.random.default_rng(21)
+    xh = host_rows(rng.standard_normal((33, 256)), dtype)
+    x64 = promote(xh, dtype)
+    code = harp.HARP_F32 if dtype == "f32" else harp.HARP_BF16
+    for n in (2, 3):
+        for tr in (False, True):
+            x = to_device(xh, dtype)
+            harp.harp_apply_passes(plans[:n], x.data_ptr(), 33, code, tr, torch.cuda.current_stream().cuda_stream)
+            want = orc.transpose_passes(oplans[:n], x64) if tr else orc.forward_passes(oplans[:n], x64)
+            assert orc.rel_err_rows(to_host_f64(x), want) <= n * TOL[dtype]
+    with pytest.raises(harp.HarpError):
+        harp.harp_apply_passes([plans[0], harp.plan_from_spec(wl.tiny_plan(1, (4, 4), kind="qr"))],
+                               to_device(xh, dtype).data_ptr(), 33, code)

@@ -61,6 +61,25 @@ def test_forward_and_transpose_equal_dense_product(radices):
     assert np.allclose(orc.dense(plan), Q, atol=1e-12, rtol=0)
 
 
+def test_passes_compose_as_a_product_of_dense_matrices():
+    """Several passes: forward is x Q_0 Q_1 Q_2 with each Q_k built independently from its own
+    stages; the transpose is the inverse, applied in the opposite order."""
+    specs = [wl.tiny_plan(3, (4, 2, 3), kind="qr", perm="random", signs=True),
+             wl.tiny_plan(4, (3, 8), kind="qr", perm="identity", signs=False),
+             wl.tiny_plan(5, (2, 2, 6), kind="qr", perm="random", signs=False)]
+    plans = [orc.OraclePlan.from_spec(sp) for sp in specs]
+    Qs = [dense_Q(sp) for sp in specs]
+    x = np.random.default_rng(2).standard_normal((4, 24))
+    assert np.allclose(orc.forward_passes(plans, x), x @ Qs[0] @ Qs[1] @ Qs[2], atol=1e-12, rtol=0)
+    assert np.allclose(orc.transpose_passes(plans, x), x @ Qs[2].T @ Qs[1].T @ Qs[0].T, atol=1e-12, rtol=0)
+    # (the blocks are orthogonal to fp32 rounding only)
+    assert np.allclose(orc.transpose_passes(plans, orc.forward_passes(plans, x)), x, atol=1e-5, rtol=0)
+    # the order matters: the passes do not commute
+    assert not np.allclose(orc.forward_passes(plans[::-1], x), orc.forward_passes(plans, x), atol=1e-6)
+    # one pass is the plain apply
+    assert np.array_equal(orc.forward_passes(plans[:1], x), orc.forward(plans[0], x))
+
+
 @pytest.mark.parametrize("radices", TINY)
 def test_orthogonality_dense(radices):
     plan = orc.OraclePlan.from_spec(wl.tiny_plan(3, radices))
