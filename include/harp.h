@@ -194,6 +194,25 @@ harp_status_t harp_apply_two_sided_static(void *W, harp_dtype_t dtype,
 /* Capacity in bytes of the fixed scratch array used by harp_apply_two_sided_static. */
 int64_t harp_two_sided_static_capacity_bytes(void);
 
+/* ---- Gradient with respect to the block kernels (what Algorithm 3 needs from the apply; the
+ * gradient with respect to the rows is harp_apply with transpose = 1 on dL/dy) ----------------
+ * For y = x Q (harp_apply, transpose = 0) and a scalar loss L with G = dL/dy:
+ *   dL/dK_t[c][i][j] = sum over rows of v_t[base_c + i s_t] * g_{t+1}[base_c + j s_t],
+ * v_t the input of stage t in the forward pass and g_{t+1} = dL/d(output of stage t)
+ * (g_m = G, g_t = g_{t+1} M_t^T) -- the chain rule through Algorithm 1.
+ *   x, gy      DEVICE n_rows x d of dtype, read only
+ *   grad       DEVICE float[harp_plan_n_params(plan)], laid out like the blocks given to
+ *              harp_plan_create (stage after stage, [D_t][b_t][b_t]); overwritten, or added to
+ *              if accumulate != 0
+ * Any schedule is accepted.  Sums over rows are taken in fp64 by one thread per entry (no
+ * atomics: the result does not depend on scheduling).  The call allocates and frees scratch
+ * on the stream (at most ~256 MB); HARP_ERR_ALLOC if that fails.  Asynchronous on stream. */
+harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x, const void *gy, int64_t n_rows,
+                               harp_dtype_t dtype, float *grad, int accumulate, void *stream);
+
+/* Number of block-kernel entries of the plan: sum over stages of d * b_t (-1 for NULL). */
+int64_t harp_plan_n_params(const harp_plan_t *plan);
+
 /* ---- Diagnostics of a processed layer (appendix "Incoherence diagnostics") ----------------
  * One pass over a row-major DEVICE matrix each; asynchronous on stream; nothing is allocated.
  * out is a DEVICE array of four doubles, 8-byte aligned, owned by the caller: out[0] receives

@@ -122,6 +122,35 @@ def two_sided(plan_out: OraclePlan, plan_in: OraclePlan, w: np.ndarray) -> np.nd
     return forward(plan_out, rows_done.T).T                     # each column . Q_out
 
 
+def grad_blocks(plan: OraclePlan, x: np.ndarray, gy: np.ndarray) -> List[np.ndarray]:
+    """dL/dK_t for y = forward(x) and G = dL/dy (chain rule through Algorithm 1):
+    g_m = G, g_t = g_{t+1} M_t^T, dL/dK_t[c][i][j] = sum_rows v_t[base_c + i s_t] g_{t+1}[base_c + j s_t],
+    with v_t the input of stage t.  Returns one array [D_t][b_t][b_t] per stage."""
+    v = np.array(x, dtype=np.float64, ndmin=2)
+    if plan.signs is not None:
+        v = v * plan.signs[None, :]
+    if plan.perm is not None:
+        v = v[:, plan.perm]
+    n = v.shape[0]
+    states, strides = [], []
+    s = 1
+    for t, b in enumerate(plan.radices):
+        states.append(v)                                       # v_t: what stage t reads
+        strides.append(s)
+        v = _stage(v, b, s, plan.blocks[t], transposed=False)
+        s *= b
+    g = np.array(gy, dtype=np.float64, ndmin=2)
+    grads: List[np.ndarray] = [np.zeros(0)] * len(plan.radices)
+    for t in range(len(plan.radices) - 1, -1, -1):
+        b, s = plan.radices[t], strides[t]
+        grp = plan.d // (b * s)
+        vt = states[t].reshape(n, grp, b, s)                   # [row][alpha][i][beta]
+        gt = g.reshape(n, grp, b, s)                           # [row][alpha][j][beta]
+        grads[t] = np.einsum("naib,najb->abij", vt, gt).reshape(grp * s, b, b)   # block c = alpha*s + beta
+        g = _stage(g, b, s, plan.blocks[t], transposed=True)   # gradient with respect to v_t
+    return grads
+
+
 def forward_passes(plans: Sequence[OraclePlan], x: np.ndarray) -> np.ndarray:
     """Several passes (Section "HARP processors"): y = x . Q_0 . Q_1 ... , each Q_k one processor."""
     y = np.array(x, dtype=np.float64, ndmin=2)

@@ -67,6 +67,10 @@ def lib() -> ctypes.CDLL:
         L.harp_apply_two_sided_static.argtypes = [vp, ctypes.c_int, vp, vp, vp]
         L.harp_two_sided_static_capacity_bytes.restype = i64
         L.harp_two_sided_static_capacity_bytes.argtypes = []
+        L.harp_grad_blocks.restype = ctypes.c_int
+        L.harp_grad_blocks.argtypes = [vp, vp, vp, i64, ctypes.c_int, vp, ctypes.c_int, vp]
+        L.harp_plan_n_params.restype = i64
+        L.harp_plan_n_params.argtypes = [vp]
         L.harp_weight_incoherence.restype = ctypes.c_int
         L.harp_weight_incoherence.argtypes = [vp, i64, i64, ctypes.c_int, vp, vp]
         L.harp_offblock_energy.restype = ctypes.c_int
@@ -250,6 +254,19 @@ def harp_two_sided_static_capacity_bytes() -> int:
 
 def harp_two_sided_scratch_bytes(plan_out: Plan, plan_in: Plan, dtype: int) -> int:
     return int(lib().harp_two_sided_scratch_bytes(plan_out.handle, plan_in.handle, int(dtype)))
+
+
+def harp_plan_n_params(plan: Plan) -> int:
+    return int(lib().harp_plan_n_params(plan.handle))
+
+
+def harp_grad_blocks(plan: Plan, x_ptr: int, gy_ptr: int, n_rows: int, dtype: int, grad_ptr: int,
+                     accumulate: bool = False, stream: int = 0) -> None:
+    """dL/d(block kernels) for y = x Q and G = dL/dy; grad_ptr: DEVICE float[harp_plan_n_params(plan)]."""
+    st = lib().harp_grad_blocks(plan.handle, x_ptr, gy_ptr, int(n_rows), int(dtype), grad_ptr,
+                                1 if accumulate else 0, stream or None)
+    if st != HARP_OK:
+        raise HarpError(st, "harp_grad_blocks")
 
 
 def harp_weight_incoherence(a_ptr: int, m: int, n: int, dtype: int, out_ptr: int, stream: int = 0) -> None:

@@ -1,0 +1,91 @@
+"""harp_grad_blocks on the GPU against the oracle's chain rule, and against invariants at a
+configuration's full dimension."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2605_29843_b200 as harp
+from oracle import harp_oracle as orc
+from paper_2605_29843_b200 import workloads as wl
+from harp_testlib import host_rows, promote, to_device
+
+pytestmark = pytest.mark.gpu
+
+DT = {"f32": harp.HARP_F32, "bf16": harp.HARP_BF16}
+
+
+def _gpu_grad(plan, xh, gh, dtype, accumulate=False, init=None):
+    n = xh.shape[0]
+    x_d, g_d = to_device(xh, dtype), to_device(gh, dtype)
+    n_par = harp.harp_plan_n_params(plan)
+    out = torch.full((n_par,), 3.0, dtype=torch.float32, device="cuda") if init is None else init.clone()
+    harp.harp_grad_blocks(plan, x_d.data_ptr(), g_d.data_ptr(), n, DT[dtype], out.data_ptr(), accumulate,
+                          torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    return out.cpu().numpy().astype(np.float64), x_d, g_d
+
+
+def _flat(grads):
+    return np.concatenate([g.ravel() for g in grads])
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("radices,perm", [((4,), "identity"), ((2, 2, 2), "random"), ((4, 3, 5), "random"),
+                                          ((16, 8, 2), "identity"), ((7, 2), "random"), ((43, 2), "identity")])
+def test_grad_blocks_matches_the_oracle(dtype, radices, perm):
+    spec = wl.tiny_plan(31, radices, kind="qr", perm=perm, signs=True)
+    plan = harp.plan_from_spec(spec)
+    oplan = orc.OraclePlan.from_spec(spec)
+    rng = np.random.default_rng(32)
+    xh = host_rows(rng.standard_normal((29, spec.d)), dtype)
+    gh = host_rows(rng.standard_normal((29, spec.d)), dtype)
+    got, x_d, g_d = _gpu_grad(plan, xh, gh, dtype)
+    want = _flat(orc.grad_blocks(oplan, promote(xh, dtype), promote(gh, dtype)))
+    assert got.shape == want.shape == (harp.harp_plan_n_params(plan),)
+    # fp32 stage states, fp64 row sums: error relative to the size of the largest entry
+    assert np.max(np.abs(got - want)) <= 2e-5 * np.max(np.abs(want))
+    # the inputs are not modified
+    assert np.array_equal(x_d.cpu().view(torch.int16 if dtype == "bf16" else torch.int32).numpy(),
+                          to_device(xh, dtype).cpu().view(torch.int16 if dtype == "bf16" else torch.int32).numpy())
+
+
+def test_accumulate_and_row_chunks_add_up():
+    spec = wl.tiny_plan(33, (4, 4, 2), kind="qr", perm="random", signs=True)
+    plan = harp.plan_from_spec(spec)
+    rng = np.random.default_rng(34)
+    xh, gh = host_rows(rng.standard_normal((40, 32)), "f32"), host_rows(rng.standard_normal((40, 32)), "f32")
+    full, _, _ = _gpu_grad(plan, xh, gh, "f32")
+    first, _, _ = _gpu_grad(plan, xh[:15], gh[:15], "f32")
+    both, _, _ = _gpu_grad(plan, xh[15:], gh[15:], "f32", accumulate=True,
+                           init=torch.from_numpy(first.astype(np.float32)).cuda())
+    assert np.max(np.abs(both - full)) <= 1e-5 * np.max(np.abs(full))
+    # no rows: the result is zero (or untouched when accumulating)
+    n_par = harp.harp_plan_n_params(plan)
+    out = torch.full((n_par,), 3.0, dtype=torch.float32, device="cuda")
+    harp.harp_grad_blocks(plan, 0, 0, 0, harp.HARP_F32, out.data_ptr())
+    assert float(out.abs().max()) == 0.0
+
+
+def test_euler_identity_at_full_dimension():
+    """cfg2's plan (d = 4096, six radix-4 stages, digit-reversal permutation): y is homogeneous of
+    degree one in the kernels of every stage, so <K_t, dL/dK_t> = sum(y * G) for each t; y comes
+    from harp_apply itself."""
+    w = wl.config(2)
+    spec = w.plans["q"]
+    plan = harp.plan_from_spec(spec)
+    n = 512
+    g = torch.Generator(device="cuda").manual_seed(7)
+    x = torch.randn((n, spec.d), device="cuda", generator=g)
+    G = torch.randn((n, spec.d), device="cuda", generator=g)
+    grad = torch.zeros(harp.harp_plan_n_params(plan), dtype=torch.float32, device="cuda")
+    harp.harp_grad_blocks(plan, x.data_ptr(), G.data_ptr(), n, harp.HARP_F32, grad.data_ptr())
+    y = x.clone()
+    harp.apply_(plan, y)
+    L = float((y.double() * G.double()).sum())
+    off = 0
+    for t, b in enumerate(spec.radices):
+        k = torch.from_numpy(np.ascontiguousarray(spec.blocks[t], dtype=np.float32)).cuda().flatten()
+        got = float((k.double() * grad[off:off + k.numel()].double()).sum())
+        off += k.numel()
+        assert got == pytest.approx(L, rel=2e-4), t
+    assert off == grad.numel()
