@@ -31,7 +31,6 @@
 // permutations use the generic kernel.
 #include <algorithm>
 #include <cmath>
-#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <map>
@@ -224,30 +223,14 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
                     }
                 }
             } else if ((MODES & bit(MODE_SS)) && ph.mode == MODE_SS && ph.B == 16) {
-                // software pipeline over this warp's items: operands of the next item are in
-                // flight while the current one is multiplied
-                uint4 rawA[4][2], rawB[4][2], bfA[8], bfB[8];
+                // (prefetching the next item's operands or fragments in registers was measured: the
+                // kernel sits at the register limit and every variant that holds more spills)
+                uint4 raw[4][2], bf[8];
                 uint32_t unused[8][4];
-                int it = warp;
-                {
-                    for (; it < n; it += NW) {
-                        ss16_load(c, ph, it, rawA, bfA);
-                        octet_mma16<true>(rawA, bfA, unused);
-                        ss16_store(c, ph, it, rawA);
-                    }
-                }
-                if (false && it < n) ss16_load(c, ph, it, rawA, bfA);
-                while (false && it < n) {
-                    const int it2 = it + NW;
-                    if (it2 < n) ss16_load(c, ph, it2, rawB, bfB);
-                    octet_mma16<true>(rawA, bfA, unused);
-                    ss16_store(c, ph, it, rawA);
-                    if (it2 >= n) break;
-                    const int it3 = it2 + NW;
-                    if (it3 < n) ss16_load(c, ph, it3, rawA, bfA);
-                    octet_mma16<true>(rawB, bfB, unused);
-                    ss16_store(c, ph, it2, rawB);
-                    it = it3;
+                for (int it = warp; it < n; it += NW) {
+                    ss16_load(c, ph, it, raw, bf);
+                    octet_mma16<true>(raw, bf, unused);
+                    ss16_store(c, ph, it, raw);
                 }
             } else if ((MODES & bit(MODE_SS)) && ph.mode == MODE_SS) {
                 const uint32_t *bf8 = reinterpret_cast<const uint32_t *>(ph.bfrag);
@@ -271,28 +254,12 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
                     }
                 }
             } else if ((MODES & bit(MODE_GS)) && ph.mode == MODE_GS) {
-                uint4 rawA[4][2], rawB[4][2], bfA[8], bfB[8];
+                uint4 raw[4][2], bf[8];
                 uint32_t mats[8][4];
-                int it = warp;
-                {
-                    for (; it < n; it += NW) {
-                        gs_load(c, ph, it, rawA, bfA);
-                        octet_mma16<false>(rawA, bfA, mats);
-                        gs_store(c, ph, it, mats);
-                    }
-                }
-                if (false && it < n) gs_load(c, ph, it, rawA, bfA);
-                while (false && it < n) {
-                    const int it2 = it + NW;
-                    if (it2 < n) gs_load(c, ph, it2, rawB, bfB);
-                    octet_mma16<false>(rawA, bfA, mats);
+                for (int it = warp; it < n; it += NW) {
+                    gs_load(c, ph, it, raw, bf);
+                    octet_mma16<false>(raw, bf, mats);
                     gs_store(c, ph, it, mats);
-                    if (it2 >= n) break;
-                    const int it3 = it2 + NW;
-                    if (it3 < n) gs_load(c, ph, it3, rawA, bfA);
-                    octet_mma16<false>(rawB, bfB, mats);
-                    gs_store(c, ph, it2, mats);
-                    it = it3;
                 }
             } else if ((MODES & bit(MODE_PO)) && ph.mode == MODE_PO) {
                 // contiguous blocks in (ldmatrix), eight-block runs out to the same sixteen 16-byte
