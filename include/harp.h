@@ -246,9 +246,10 @@ harp_status_t harp_diag_weighted_error(const void *Wt, const void *Wq, int64_t d
                                        double *out, void *stream);
 
 /* Apply to rows that live in HOST memory (pinned memory gives full copy speed):
- * copies chunks host->device, applies, copies back, on two internal streams so that
- * copies overlap kernels; returns after the last copy has completed.  The device staging
- * buffers belong to the plan and are created at the first call.
+ * copies chunks of 16 MiB host->device, applies, copies back, on four internal streams so
+ * that copies in both directions overlap each other and the kernels; returns after the last
+ * copy has completed.  The device staging buffers (four) belong to the plan and are created at
+ * the first call.
  *   x_host   HOST n_rows x d, overwritten with the result */
 harp_status_t harp_apply_host(harp_plan_t *plan, void *x_host, int64_t n_rows,
                               harp_dtype_t dtype, int transpose);

@@ -1,6 +1,7 @@
 // C ABI of libharp.so: plan construction and validation, dispatch, two-sided
 // processing, the host-buffer pipeline.
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -149,7 +150,7 @@ extern "C" void harp_plan_destroy(harp_plan_t *p) {
         harp_fast_destroy(p);
         harp_split_destroy(p);
         harp_col_destroy(p);
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < harp_plan::kStages; ++i) {
             if (p->stage_stream[i]) { cudaStreamSynchronize(p->stage_stream[i]); cudaStreamDestroy(p->stage_stream[i]); }
             if (p->stage_buf[i]) cudaFree(p->stage_buf[i]);
         }
@@ -257,31 +258,33 @@ extern "C" harp_status_t harp_apply_host(harp_plan_t *plan, void *x_host, int64_
     DeviceGuard g(plan->device);
     if (!g.ok) return HARP_ERR_CUDA;
     const int64_t row_bytes = plan->d * (int64_t)harp_dtype_size(dtype);
-    const int64_t want = 32ll << 20;                       // staging bytes per buffer
+    // staging bytes per buffer: small enough that the first copy in and the last copy out, which
+    // nothing overlaps, are a small part of the transfer; HARP_STAGE_MB overrides (for tuning)
+    const int64_t want = (int64_t)(getenv("HARP_STAGE_MB") ? std::max(1, atoi(getenv("HARP_STAGE_MB"))) : 16) << 20;
     int64_t chunk_rows = std::max<int64_t>(1, want / row_bytes);
     const int64_t need = chunk_rows * row_bytes;
     if (plan->stage_bytes < need) {
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < harp_plan::kStages; ++i) {
             if (plan->stage_buf[i]) { cudaFree(plan->stage_buf[i]); plan->stage_buf[i] = nullptr; }
             if (cudaMalloc(&plan->stage_buf[i], (size_t)need) != cudaSuccess) { cudaGetLastError(); plan->stage_bytes = 0; return HARP_ERR_ALLOC; }
         }
         plan->stage_bytes = need;
     }
-    for (int i = 0; i < 2; ++i)
+    for (int i = 0; i < harp_plan::kStages; ++i)
         if (!plan->stage_stream[i] && cudaStreamCreateWithFlags(&plan->stage_stream[i], cudaStreamNonBlocking) != cudaSuccess)
             return HARP_ERR_CUDA;
     harp_status_t st = HARP_OK;
     int k = 0;
     for (int64_t r = 0; r < n_rows && st == HARP_OK; r += chunk_rows, ++k) {
         const int64_t rows = std::min(chunk_rows, n_rows - r);
-        const int b = k & 1;
+        const int b = k % harp_plan::kStages;
         char *h = static_cast<char *>(x_host) + r * row_bytes;
         cudaStream_t s = plan->stage_stream[b];
         if (cudaMemcpyAsync(plan->stage_buf[b], h, (size_t)(rows * row_bytes), cudaMemcpyHostToDevice, s) != cudaSuccess) st = HARP_ERR_CUDA;
         if (st == HARP_OK) st = harp_apply(plan, plan->stage_buf[b], rows, dtype, transpose, s);
         if (st == HARP_OK && cudaMemcpyAsync(h, plan->stage_buf[b], (size_t)(rows * row_bytes), cudaMemcpyDeviceToHost, s) != cudaSuccess) st = HARP_ERR_CUDA;
     }
-    for (int i = 0; i < 2; ++i)
+    for (int i = 0; i < harp_plan::kStages; ++i)
         if (cudaStreamSynchronize(plan->stage_stream[i]) != cudaSuccess && st == HARP_OK) st = HARP_ERR_CUDA;
     return st;
 }

@@ -48,9 +48,10 @@ struct harp_plan {
     SplitPlan *split = nullptr;
     ColPlan *col = nullptr;
     // staging owned by harp_apply_host
-    void *stage_buf[2] = {nullptr, nullptr};
+    static constexpr int kStages = 4;
+    void *stage_buf[kStages] = {nullptr, nullptr, nullptr, nullptr};
     int64_t stage_bytes = 0;
-    cudaStream_t stage_stream[2] = {nullptr, nullptr};
+    cudaStream_t stage_stream[kStages] = {nullptr, nullptr, nullptr, nullptr};
 };
 
 extern std::atomic<int64_t> g_harp_launches;
