@@ -72,6 +72,25 @@ def test_null_arguments():
     assert harp.harp_launch_count() >= 0
 
 
+def test_null_arguments_of_the_widened_entry_points():
+    """Passes, gradient and diagnostics reject bad arguments before any CUDA call."""
+    L = harp.lib()
+    assert L.harp_apply_passes(None, 1, None, 4, 0, 0, None) == 1
+    arr = (ctypes.c_void_p * 1)(None)
+    assert L.harp_apply_passes(arr, 1, None, 4, 0, 0, None) == 1          # a NULL plan in the list
+    assert L.harp_apply_passes(arr, 0, None, 4, 0, 0, None) == 3          # no passes
+    assert L.harp_grad_blocks(None, None, None, 4, 0, None, 0, None) == 1
+    assert L.harp_plan_n_params(None) == -1
+    buf = (ctypes.c_double * 4)()
+    assert L.harp_weight_incoherence(None, 4, 4, 0, buf, None) == 1
+    assert L.harp_weight_incoherence(buf, 0, 4, 0, buf, None) == 2        # empty matrix
+    assert L.harp_weight_incoherence(buf, 4, 4, 7, buf, None) == 6        # unknown dtype
+    assert L.harp_offblock_energy(None, 4, 2, 0, buf, None) == 1
+    assert L.harp_offblock_energy(buf, 4, 5, 0, buf, None) == 2           # block larger than n
+    assert L.harp_offblock_energy(buf, 4, 0, 0, buf, None) == 2
+    assert L.harp_diag_weighted_error(None, buf, 2, 2, 0, buf, 0, buf, None) == 1
+
+
 def test_no_gpu_means_an_error_not_a_fallback():
     import torch
     if torch.cuda.is_available():
