@@ -6,10 +6,16 @@
 // y = v_m.  With G = dL/dy:   g_m = G,   g_t = g_{t+1} M_t^T,
 //     dL/dK_t[c][i][j] = sum over rows of  v_t[base_c + i s_t] * g_{t+1}[base_c + j s_t].
 //
-// This first version favours clarity over speed: the rows are processed in chunks; for a chunk
-// all forward states v_0..v_{m-1} are kept in global scratch (fp32), the gradient state is walked
-// back stage by stage, and every entry of the result is owned by one thread that sums over the
-// chunk's rows in fp64 in a fixed order -- no atomics, so the result does not depend on scheduling.
+// The rows are processed in chunks; for a chunk all forward states v_0..v_{m-1} are kept in global
+// scratch (fp32) and the gradient state is walked back stage by stage.  Every sum over rows is
+// taken in fp64 in a fixed order -- no atomics, so the result does not depend on scheduling.
+//
+// Stages of radix 2, 4 and 8 run in "block owner" kernels: a thread owns one block c of the stage,
+// keeps K_t[c] in registers and walks the rows of its slice of the chunk, so neighbouring lanes
+// read neighbouring coordinates (or one vector when s_t = 1) and K is read once.  The backward
+// kernel of such a stage does both jobs in one sweep over v_t and g_{t+1}: it writes g_t and adds
+// v_t[i] g_{t+1}[j] into its B x B fp64 accumulators; the per-slice sums are then added slice by
+// slice.  Other radices use the plain one-thread-per-element kernels below them.
 #include <algorithm>
 
 #include "harp_internal.h"
@@ -21,6 +27,189 @@ constexpr int kThreads = 256;
 template <typename T> __device__ __forceinline__ float to_f32(T v);
 template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
 template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+constexpr int kOwnThreads = 128;   // block-owner kernels: blocks per CTA
+constexpr int kFwdSliceRows = 8;   //                      rows per CTA, forward
+constexpr int kBwdSliceRows = 16;  //                      rows per CTA (one set of partial sums), backward
+constexpr int kRowBatch = 4;       //                      rows whose loads are issued together
+
+template <int B> __device__ __forceinline__ void load_block(const float *p, int64_t s, float (&v)[B]) {
+    if (s == 1) {
+        if constexpr (B == 2) {
+            const float2 a = *reinterpret_cast<const float2 *>(p);
+            v[0] = a.x; v[1] = a.y;
+        } else {
+#pragma unroll
+            for (int q = 0; q < B / 4; ++q) {
+                const float4 a = reinterpret_cast<const float4 *>(p)[q];
+                v[4 * q] = a.x; v[4 * q + 1] = a.y; v[4 * q + 2] = a.z; v[4 * q + 3] = a.w;
+            }
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < B; ++i) v[i] = p[(int64_t)i * s];
+    }
+}
+
+template <int B> __device__ __forceinline__ void store_block(float *p, int64_t s, const float (&v)[B]) {
+    if (s == 1) {
+        if constexpr (B == 2) {
+            *reinterpret_cast<float2 *>(p) = make_float2(v[0], v[1]);
+        } else {
+#pragma unroll
+            for (int q = 0; q < B / 4; ++q)
+                reinterpret_cast<float4 *>(p)[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < B; ++i) p[(int64_t)i * s] = v[i];
+    }
+}
+
+// forward stage, block owner: out[r][base_c + j s] = sum_i in[r][base_c + i s] K[c][i][j]
+template <int B>
+__global__ void __launch_bounds__(kOwnThreads)
+fwd_owner_kernel(const float *__restrict__ in, float *__restrict__ out, int64_t rows, int64_t d, int64_t s,
+                 const float *__restrict__ K) {
+    const int64_t c = (int64_t)blockIdx.x * kOwnThreads + threadIdx.x;
+    if (c >= d / B) return;
+    float k[B][B];
+#pragma unroll
+    for (int i = 0; i < B; ++i)
+#pragma unroll
+        for (int j = 0; j < B; ++j) k[i][j] = K[c * (B * B) + i * B + j];
+    const int64_t alpha = c / s, base = alpha * B * s + (c - alpha * s);
+    const int64_t r0 = (int64_t)blockIdx.y * kFwdSliceRows, r1 = min(rows, r0 + kFwdSliceRows);
+    for (int64_t r = r0; r < r1; r += kRowBatch) {
+        float v[kRowBatch][B];
+#pragma unroll
+        for (int u = 0; u < kRowBatch; ++u)
+            if (r + u < r1) load_block<B>(in + (r + u) * d + base, s, v[u]);
+#pragma unroll
+        for (int u = 0; u < kRowBatch; ++u) {
+            if (r + u >= r1) break;
+            float o[B];
+#pragma unroll
+            for (int j = 0; j < B; ++j) {
+                float acc = 0.f;
+#pragma unroll
+                for (int i = 0; i < B; ++i) acc = fmaf(v[u][i], k[i][j], acc);
+                o[j] = acc;
+            }
+            store_block<B>(out + (r + u) * d + base, s, o);
+        }
+    }
+}
+
+// backward stage, block owner: g_out[r][base_c + i s] = sum_j g[r][base_c + j s] K[c][i][j] (when
+// g_out is given) and part[slice][i B + j][c] = sum over the slice's rows of v[..i..] g[..j..].
+template <int B>
+__global__ void __launch_bounds__(kOwnThreads)
+bwd_owner_kernel(const float *__restrict__ v, const float *__restrict__ g, float *__restrict__ g_out, int64_t rows,
+                 int64_t d, int64_t s, const float *__restrict__ K, double *__restrict__ part) {
+    const int64_t nblk = d / B;
+    const int64_t c = (int64_t)blockIdx.x * kOwnThreads + threadIdx.x;
+    if (c >= nblk) return;
+    float k[B][B];
+    double acc[B][B];
+#pragma unroll
+    for (int i = 0; i < B; ++i)
+#pragma unroll
+        for (int j = 0; j < B; ++j) {
+            k[i][j] = K[c * (B * B) + i * B + j];
+            acc[i][j] = 0.0;
+        }
+    const int64_t alpha = c / s, base = alpha * B * s + (c - alpha * s);
+    constexpr int U = B == 8 ? 2 : kRowBatch;         // radix 8 already fills the register file
+    const int64_t r0 = (int64_t)blockIdx.y * kBwdSliceRows, r1 = min(rows, r0 + kBwdSliceRows);
+    for (int64_t r = r0; r < r1; r += U) {
+        float vv[U][B], gg[U][B];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (r + u < r1) {
+                load_block<B>(v + (r + u) * d + base, s, vv[u]);
+                load_block<B>(g + (r + u) * d + base, s, gg[u]);
+            }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (r + u >= r1) break;
+#pragma unroll
+            for (int i = 0; i < B; ++i)
+#pragma unroll
+                for (int j = 0; j < B; ++j) acc[i][j] += (double)vv[u][i] * (double)gg[u][j];
+            if (g_out) {
+                float o[B];
+#pragma unroll
+                for (int i = 0; i < B; ++i) {
+                    float a = 0.f;
+#pragma unroll
+                    for (int j = 0; j < B; ++j) a = fmaf(gg[u][j], k[i][j], a);
+                    o[i] = a;
+                }
+                store_block<B>(g_out + (r + u) * d + base, s, o);
+            }
+        }
+    }
+    double *dst = part + (int64_t)blockIdx.y * (B * B) * nblk + c;
+#pragma unroll
+    for (int i = 0; i < B; ++i)
+#pragma unroll
+        for (int j = 0; j < B; ++j) dst[(int64_t)(i * B + j) * nblk] = acc[i][j];
+}
+
+// grad[c][i][j] (+)= sum over slices of part[slice][i b + j][c].  A CTA owns 32 neighbouring
+// entries (one per lane); warp w adds the slices w, w + 8, ... and the eight sums are added in
+// the order of w, so the result does not depend on scheduling.
+__global__ void __launch_bounds__(kThreads)
+reduce_slices_kernel(const double *__restrict__ part, int64_t n_slices, int64_t nblk, int bb, float *__restrict__ grad,
+                     int accumulate) {
+    __shared__ double warp_sum[kThreads / 32][32];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int64_t total = nblk * bb;
+    for (int64_t q0 = (int64_t)blockIdx.x * 32; q0 < total; q0 += (int64_t)gridDim.x * 32) {
+        const int64_t q = q0 + lane;
+        double sum = 0.0;
+        if (q < total) {
+#pragma unroll 4
+            for (int64_t sl = w; sl < n_slices; sl += kThreads / 32) sum += part[sl * total + q];
+        }
+        warp_sum[w][lane] = sum;
+        __syncthreads();
+        if (w == 0 && q < total) {
+            double all = warp_sum[0][lane];
+            for (int k = 1; k < kThreads / 32; ++k) all += warp_sum[k][lane];
+            const int64_t ij = q / nblk, c = q - ij * nblk;
+            float *dst = grad + c * bb + ij;
+            *dst = accumulate ? *dst + (float)all : (float)all;
+        }
+        __syncthreads();
+    }
+}
+
+// position of element i in the staged row of load_rows_kernel: two elements of padding per 64,
+// so that a digit-reversal gather (strides of 64 elements and more) spreads over the banks
+__device__ __forceinline__ int64_t staged_pos(int64_t i) { return i + 2 * (i >> 6); }
+
+// as load_kernel, one CTA per row: the row of x is read in order into shared memory and gathered
+// from there, so the permutation costs no scattered global reads
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+load_rows_kernel(const T *__restrict__ x, const T *__restrict__ gy, int64_t rows, int64_t d, const int32_t *__restrict__ perm,
+                 const int8_t *__restrict__ signs, float *__restrict__ v0, float *__restrict__ g) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    T *row = reinterpret_cast<T *>(smem_raw);
+    for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
+        for (int64_t i = threadIdx.x; i < d; i += kThreads) row[staged_pos(i)] = x[r * d + i];
+        __syncthreads();
+        for (int64_t i = threadIdx.x; i < d; i += kThreads) {
+            const int64_t src = perm[i];
+            const float sg = (signs && signs[src] < 0) ? -1.f : 1.f;
+            v0[r * d + i] = sg * to_f32<T>(row[staged_pos(src)]);
+            g[r * d + i] = to_f32<T>(gy[r * d + i]);
+        }
+        __syncthreads();
+    }
+}
 
 // v0[r][i] = s[perm[i]] * x[r][perm[i]],  g[r][i] = gy[r][i]   (both fp32)
 template <typename T>
@@ -90,6 +279,39 @@ unsigned grid_for(int64_t work) {
     return (unsigned)std::max<int64_t>(1, std::min<int64_t>((work + kThreads - 1) / kThreads, 148 * 16));
 }
 
+bool owner_radix(int b) { return b == 2 || b == 4 || b == 8; }
+
+dim3 owner_grid(int64_t d, int b, int64_t rows, int slice_rows) {
+    return dim3((unsigned)((d / b + kOwnThreads - 1) / kOwnThreads), (unsigned)((rows + slice_rows - 1) / slice_rows));
+}
+
+void launch_fwd_owner(int b, const float *in, float *out, int64_t rows, int64_t d, int64_t s, const float *K, cudaStream_t st) {
+    const dim3 grid = owner_grid(d, b, rows, kFwdSliceRows);
+    if (b == 2) fwd_owner_kernel<2><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K);
+    else if (b == 4) fwd_owner_kernel<4><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K);
+    else fwd_owner_kernel<8><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K);
+}
+
+void launch_bwd_owner(int b, const float *v, const float *g, float *g_out, int64_t rows, int64_t d, int64_t s, const float *K,
+                      double *part, cudaStream_t st) {
+    const dim3 grid = owner_grid(d, b, rows, kBwdSliceRows);
+    if (b == 2) bwd_owner_kernel<2><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part);
+    else if (b == 4) bwd_owner_kernel<4><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part);
+    else bwd_owner_kernel<8><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part);
+}
+
+template <typename T>
+void launch_load(const T *x, const T *gy, int64_t rows, int64_t d, const harp_plan_t *plan, float *v0, float *g, cudaStream_t st) {
+    const size_t smem = (size_t)(d + 2 * (d >> 6) + 2) * sizeof(T);
+    static const bool big_ok =
+        cudaFuncSetAttribute(load_rows_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) == cudaSuccess;
+    if (plan->d_perm && (smem <= 48 * 1024 || (big_ok && smem <= 200 * 1024)))
+        load_rows_kernel<T><<<(unsigned)std::min<int64_t>(rows, 148 * 8), kThreads, smem, st>>>(x, gy, rows, d, plan->d_perm,
+                                                                                                 plan->d_signs, v0, g);
+    else
+        load_kernel<T><<<grid_for(rows * d), kThreads, 0, st>>>(x, gy, rows, d, plan->d_perm, plan->d_signs, v0, g);
+}
+
 }  // namespace
 
 extern "C" int64_t harp_plan_n_params(const harp_plan_t *plan) { return plan ? plan->n_params : -1; }
@@ -110,42 +332,62 @@ extern "C" harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x
         if (!accumulate && cudaMemsetAsync(grad, 0, sizeof(float) * (size_t)plan->n_params, st) != cudaSuccess) return HARP_ERR_CUDA;
         return HARP_OK;
     }
-    // chunk of rows whose m forward states and one gradient state (+ one spare) fit ~256 MB
-    const int64_t per_row = (int64_t)(m + 2) * d * (int64_t)sizeof(float);
-    const int64_t chunk = std::max<int64_t>(1, std::min<int64_t>(n_rows, (256ll << 20) / per_row));
+    // chunk of rows whose m forward states, two gradient states and the per-slice sums of the
+    // block-owner stages (at most one state: 8 bytes x d b / 16 per row, b <= 8) fit ~256 MB
+    const int64_t per_row = (int64_t)(m + 3) * d * (int64_t)sizeof(float);
+    const int64_t chunk = std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(n_rows, 1 << 18), (256ll << 20) / per_row));
+    int max_owner_b = 0;
+    for (int t = 0; t < m; ++t)
+        if (owner_radix(plan->st.b[t])) max_owner_b = std::max(max_owner_b, plan->st.b[t]);
+    const int64_t state_bytes = (int64_t)(m + 2) * chunk * d * (int64_t)sizeof(float);
+    const int64_t part_bytes = ((chunk + kBwdSliceRows - 1) / kBwdSliceRows) * d * max_owner_b * (int64_t)sizeof(double);
     float *scratch = nullptr;
-    if (cudaMallocAsync(reinterpret_cast<void **>(&scratch), (size_t)(chunk * per_row), st) != cudaSuccess) {
+    if (cudaMallocAsync(reinterpret_cast<void **>(&scratch), (size_t)(state_bytes + 256 + part_bytes), st) != cudaSuccess) {
         cudaGetLastError();
         return HARP_ERR_ALLOC;
     }
     const int64_t plane = chunk * d;                  // floats per state
     float *ga = scratch + (int64_t)m * plane, *gb = ga + plane;
+    // fp64 per-slice sums of the block-owner stages, behind the states, on the next 256-byte boundary
+    double *part = reinterpret_cast<double *>((reinterpret_cast<uintptr_t>(gb + plane) + 255) & ~(uintptr_t)255);
     harp_status_t rc = HARP_OK;
     for (int64_t r0 = 0; r0 < n_rows && rc == HARP_OK; r0 += chunk) {
         const int64_t rows = std::min(chunk, n_rows - r0);
         const unsigned grid = grid_for(rows * d);
         if (dtype == HARP_F32)
-            load_kernel<float><<<grid, kThreads, 0, st>>>((const float *)x + r0 * d, (const float *)gy + r0 * d, rows, d,
-                                                          plan->d_perm, plan->d_signs, scratch, ga);
+            launch_load<float>((const float *)x + r0 * d, (const float *)gy + r0 * d, rows, d, plan, scratch, ga, st);
         else
-            load_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>((const __nv_bfloat16 *)x + r0 * d, (const __nv_bfloat16 *)gy + r0 * d,
-                                                                  rows, d, plan->d_perm, plan->d_signs, scratch, ga);
+            launch_load<__nv_bfloat16>((const __nv_bfloat16 *)x + r0 * d, (const __nv_bfloat16 *)gy + r0 * d, rows, d, plan, scratch,
+                                       ga, st);
+        int launches = 1;
         // forward states v_1 .. v_{m-1} (v_t in plane t)
-        for (int t = 0; t + 1 < m; ++t)
-            stage_kernel<<<grid, kThreads, 0, st>>>(scratch + t * plane, scratch + (t + 1) * plane, rows, d, plan->st.b[t],
-                                                    plan->st.s[t], plan->d_blocks + plan->st.off[t], 0);
-        // backward: entry sums, then the gradient state one stage back
-        float *g_cur = ga, *g_nxt = gb;
-        for (int t = m - 1; t >= 0; --t) {
-            outer_kernel<<<(unsigned)std::min<int64_t>((d * plan->st.b[t] + 31) / 32, 148 * 64), kThreads, 0, st>>>(scratch + t * plane, g_cur, rows, d, plan->st.b[t], plan->st.s[t],
-                                                                      grad + plan->st.off[t], (accumulate || r0 > 0) ? 1 : 0);
-            if (t > 0) {
-                stage_kernel<<<grid, kThreads, 0, st>>>(g_cur, g_nxt, rows, d, plan->st.b[t], plan->st.s[t],
-                                                        plan->d_blocks + plan->st.off[t], 1);
-                std::swap(g_cur, g_nxt);
-            }
+        for (int t = 0; t + 1 < m; ++t, ++launches) {
+            const int b = plan->st.b[t];
+            const float *K = plan->d_blocks + plan->st.off[t];
+            if (owner_radix(b)) launch_fwd_owner(b, scratch + t * plane, scratch + (t + 1) * plane, rows, d, plan->st.s[t], K, st);
+            else stage_kernel<<<grid, kThreads, 0, st>>>(scratch + t * plane, scratch + (t + 1) * plane, rows, d, b, plan->st.s[t], K, 0);
         }
-        g_harp_launches.fetch_add(1 + (m - 1) + m + (m - 1), std::memory_order_relaxed);
+        // backward: entry sums, and the gradient state one stage back
+        float *g_cur = ga, *g_nxt = gb;
+        const int acc = (accumulate || r0 > 0) ? 1 : 0;
+        for (int t = m - 1; t >= 0; --t) {
+            const int b = plan->st.b[t];
+            const int64_t s = plan->st.s[t];
+            const float *K = plan->d_blocks + plan->st.off[t];
+            if (owner_radix(b)) {
+                launch_bwd_owner(b, scratch + t * plane, g_cur, t > 0 ? g_nxt : nullptr, rows, d, s, K, part, st);
+                reduce_slices_kernel<<<(unsigned)std::min<int64_t>((d * b + 31) / 32, 148 * 16), kThreads, 0, st>>>(part, (rows + kBwdSliceRows - 1) / kBwdSliceRows, d / b, b * b,
+                                                                           grad + plan->st.off[t], acc);
+                launches += 2;
+            } else {
+                outer_kernel<<<(unsigned)std::min<int64_t>((d * b + 31) / 32, 148 * 64), kThreads, 0, st>>>(scratch + t * plane, g_cur, rows,
+                                                                                                         d, b, s, grad + plan->st.off[t], acc);
+                if (t > 0) stage_kernel<<<grid, kThreads, 0, st>>>(g_cur, g_nxt, rows, d, b, s, K, 1);
+                launches += t > 0 ? 2 : 1;
+            }
+            if (t > 0) std::swap(g_cur, g_nxt);
+        }
+        g_harp_launches.fetch_add(launches, std::memory_order_relaxed);
         if (cudaGetLastError() != cudaSuccess) rc = HARP_ERR_CUDA;
     }
     cudaFreeAsync(scratch, st);

@@ -49,6 +49,23 @@ def test_grad_blocks_matches_the_oracle(dtype, radices, perm):
                           to_device(xh, dtype).cpu().view(torch.int16 if dtype == "bf16" else torch.int32).numpy())
 
 
+@pytest.mark.parametrize("radices", [(8, 4, 2), (2, 8), (4, 4, 4)])
+def test_rows_spanning_several_slices(radices):
+    """More rows than one thread block of the block-owner kernels walks, with a ragged last slice
+    and a ragged last batch; radix 8 both at stride one and strided."""
+    spec = wl.tiny_plan(35, radices, kind="qr", perm="random", signs=True)
+    plan = harp.plan_from_spec(spec)
+    oplan = orc.OraclePlan.from_spec(spec)
+    rng = np.random.default_rng(36)
+    xh = host_rows(rng.standard_normal((71, spec.d)), "f32")
+    gh = host_rows(rng.standard_normal((71, spec.d)), "f32")
+    got, _, _ = _gpu_grad(plan, xh, gh, "f32")
+    want = _flat(orc.grad_blocks(oplan, promote(xh, "f32"), promote(gh, "f32")))
+    assert np.max(np.abs(got - want)) <= 2e-5 * np.max(np.abs(want))
+    again, _, _ = _gpu_grad(plan, xh, gh, "f32")
+    assert np.array_equal(got, again)                       # fixed summation order
+
+
 def test_accumulate_and_row_chunks_add_up():
     spec = wl.tiny_plan(33, (4, 4, 2), kind="qr", perm="random", signs=True)
     plan = harp.plan_from_spec(spec)
