@@ -62,6 +62,15 @@ struct SplitPass {
     SplitPhase ph[kMaxSplitPhases];
 };
 
+// Programmatic dependent launch: everything above this call reads only the plan's tables, so a
+// kernel launched with the stream-serialisation attribute runs it while the kernel before it in
+// the stream is still busy; the rows are touched only after that kernel has completed.  The next
+// kernel in the stream may then start its own preamble.  Without the attribute both are no-ops.
+__device__ __forceinline__ void rows_ready_barrier() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 __device__ __forceinline__ uint32_t lds32(uint32_t addr) {
     uint32_t v;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
@@ -142,6 +151,7 @@ harp_split_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_
         cp_async_commit();
     };
 
+    rows_ready_barrier();
     int buf = 0;
     if (n_buf == 2 && part < n_tiles) copy_in(part, sbase0);
     for (int64_t tile = part; tile < n_tiles; tile += n_parts) {
@@ -336,6 +346,7 @@ harp_upper_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_
     const int uo = un / lo_n, lo = un - uo * lo_n;
     const int mt_shift = MT == 4 ? 2 : (MT == 2 ? 1 : 0);
 
+    rows_ready_barrier();
     for (int64_t tile = part; tile < n_tiles; tile += n_parts) {
         const int64_t row0 = row_begin + tile * tile_rows;
         // ---- copy in, transposing: unit = (row, octet of l, octet of u)
@@ -777,6 +788,27 @@ void harp_split_destroy(harp_plan *plan) {
     plan->split = nullptr;
 }
 
+// Launch of one pass.  overlap: let the kernel's preamble run under the tail of the kernel before it
+// in the stream (see rows_ready_barrier); used for small row counts, where a pass lasts a few
+// microseconds and the preamble is a large part of it.
+template <typename PassT>
+cudaError_t launch_pass(void (*kern)(__nv_bfloat16 *, int64_t, int64_t, PassT), unsigned grid, size_t smem, cudaStream_t stream,
+                        bool overlap, __nv_bfloat16 *x, int64_t r0, int64_t r1, const PassT &P) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kSplitThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kern, x, r0, r1, P);
+}
+
+constexpr int64_t kOverlapMaxRows = 64;
+
 harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype, int transpose,
                                cudaStream_t stream) {
     const SplitPlan *sp = plan->split;
@@ -784,6 +816,7 @@ harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, h
     if ((reinterpret_cast<uintptr_t>(x) & 15u) != 0) return HARP_ERR_UNSUPPORTED;
     __nv_bfloat16 *xb = static_cast<__nv_bfloat16 *>(x);
     const bool two = sp->pass[1].present || sp->dense_upper;
+    const bool overlap = n_rows <= kOverlapMaxRows;
     for (int64_t r0 = 0; r0 < n_rows; r0 += sp->chunk_rows) {
         const int64_t r1 = std::min(n_rows, r0 + (two ? sp->chunk_rows : n_rows));
         for (int s = 0; s < (two ? 2 : 1); ++s) {
@@ -796,14 +829,15 @@ harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, h
                 int64_t parts = std::max<int64_t>(1, ((int64_t)sp->sms * per_sm) / P.n_cg);
                 parts = std::min(parts, n_tiles);
                 const unsigned grid = (unsigned)(parts * P.n_cg);
+                cudaError_t err;
                 switch (sp->up_ks) {
-                    case 1: harp_upper_kernel<1><<<grid, kSplitThreads, sp->up_smem, stream>>>(xb, r0, r1, P); break;
-                    case 2: harp_upper_kernel<2><<<grid, kSplitThreads, sp->up_smem, stream>>>(xb, r0, r1, P); break;
-                    case 3: harp_upper_kernel<3><<<grid, kSplitThreads, sp->up_smem, stream>>>(xb, r0, r1, P); break;
-                    default: harp_upper_kernel<4><<<grid, kSplitThreads, sp->up_smem, stream>>>(xb, r0, r1, P); break;
+                    case 1: err = launch_pass(harp_upper_kernel<1>, grid, sp->up_smem, stream, overlap, xb, r0, r1, P); break;
+                    case 2: err = launch_pass(harp_upper_kernel<2>, grid, sp->up_smem, stream, overlap, xb, r0, r1, P); break;
+                    case 3: err = launch_pass(harp_upper_kernel<3>, grid, sp->up_smem, stream, overlap, xb, r0, r1, P); break;
+                    default: err = launch_pass(harp_upper_kernel<4>, grid, sp->up_smem, stream, overlap, xb, r0, r1, P); break;
                 }
                 g_harp_launches.fetch_add(1, std::memory_order_relaxed);
-                if (cudaGetLastError() != cudaSuccess) return HARP_ERR_CUDA;
+                if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return HARP_ERR_CUDA;
                 continue;
             }
             const PassHost &ph = sp->pass[pi];
@@ -815,10 +849,11 @@ harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, h
             int64_t parts = std::max<int64_t>(1, ((int64_t)sp->sms * per_sm) / P.n_cg);
             parts = std::min(parts, n_tiles);
             const int64_t grid = parts * P.n_cg;
-            if (ph.has16) harp_split_kernel<true><<<(unsigned)grid, kSplitThreads, ph.smem_bytes, stream>>>(xb, r0, r1, P);
-            else harp_split_kernel<false><<<(unsigned)grid, kSplitThreads, ph.smem_bytes, stream>>>(xb, r0, r1, P);
+            const cudaError_t err =
+                ph.has16 ? launch_pass(harp_split_kernel<true>, (unsigned)grid, ph.smem_bytes, stream, overlap, xb, r0, r1, P)
+                         : launch_pass(harp_split_kernel<false>, (unsigned)grid, ph.smem_bytes, stream, overlap, xb, r0, r1, P);
             g_harp_launches.fetch_add(1, std::memory_order_relaxed);
-            if (cudaGetLastError() != cudaSuccess) return HARP_ERR_CUDA;
+            if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return HARP_ERR_CUDA;
         }
         if (!two) break;
     }
