@@ -205,6 +205,16 @@ def bench_extra_configs(torch, harp, kernel, peak):
             gbs = 2 * nbytes * iters / dt / 1e9
             res[name] = {"rows_per_s": data.n_rows * iters / dt, "GBps": gbs, "frac_of_measured_peak": gbs / peak,
                          "frac_of_8TBps": gbs / 8000.0, "us_per_launch": 1e6 * dt / iters}
+        if cfg == 2:
+            # gradient of a loss with respect to the block kernels (chain rule through Algorithm 1)
+            grad = torch.zeros(harp.harp_plan_n_params(plan), dtype=torch.float32, device="cuda")
+            stream = torch.cuda.current_stream().cuda_stream
+            gb = lambda i: harp.harp_grad_blocks(plan, bufs[0].data_ptr(), bufs[1].data_ptr(), data.n_rows, harp.HARP_BF16,
+                                                 grad.data_ptr(), False, stream)
+            for i in range(2):
+                gb(i)
+            dt = time_region(torch, gb, 5)
+            res["grad_blocks"] = {"ms": 1e3 * dt / 5, "rows_per_s": data.n_rows * 5 / dt}
         if cfg == 4:
             dec = {}
             for n in w.extra["decode_rows"]:
@@ -391,6 +401,17 @@ def run_profile_case(args):
     plan = harp.plan_from_spec(spec)
     tdt = torch.float32 if w.data["x"].dtype == "f32" else torch.bfloat16
     x = torch.randn((args.profile_rows, spec.d), generator=gen, device="cuda").to(tdt)
+    if args.profile_grad:                 # gradient with respect to the block kernels instead of the apply
+        G = torch.randn((args.profile_rows, spec.d), generator=gen, device="cuda").to(tdt)
+        grad = torch.zeros(harp.harp_plan_n_params(plan), dtype=torch.float32, device="cuda")
+        for i in range(args.profile_reps):
+            harp.harp_grad_blocks(plan, x.data_ptr(), G.data_ptr(), args.profile_rows,
+                                  harp.HARP_F32 if tdt == torch.float32 else harp.HARP_BF16, grad.data_ptr(), False,
+                                  torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        print(json.dumps({"profile_case": w.name + "_grad_blocks", "rows": args.profile_rows, "reps": args.profile_reps,
+                          "launches": harp.harp_launch_count()}))
+        return
     for i in range(args.profile_reps):
         harp.apply_(plan, x, transpose=bool(i & 1), kernel=kernel)
     torch.cuda.synchronize()
@@ -408,6 +429,7 @@ def main():
     ap.add_argument("--profile-config", type=int, default=0, help="run a small profiling case of this configuration and exit")
     ap.add_argument("--profile-rows", type=int, default=8192)
     ap.add_argument("--profile-reps", type=int, default=2)
+    ap.add_argument("--profile-grad", action="store_true", help="the profiling case calls harp_grad_blocks")
     ap.add_argument("--all-configs", action="store_true")
     ap.add_argument("--no-cpu", action="store_true", help="skip the timed CPU-oracle baseline")
     ap.add_argument("--ref-rows", type=int, default=2048)
