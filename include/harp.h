@@ -100,6 +100,17 @@ harp_status_t harp_blocks_from_theta(int32_t b, int64_t n_blocks, const float *t
                                      const int8_t *theta_q, const float *scales,
                                      const float *mixer, float *out_blocks);
 
+/* Gradient with respect to the stored parameters of one stage, given the gradient with respect to
+ * its block kernels (harp_grad_blocks, copied to the host): the chain rule through B_c = Q(theta_c) G_b
+ * (Eq. 9-11), i.e. what the parameter update of Algorithm 3 needs.  All pointers HOST; no CUDA call.
+ *   theta       float[n_blocks][n_par], the point at which the blocks were built
+ *   mixer       as in harp_blocks_from_theta
+ *   grad_blocks float[n_blocks][b][b] = dL/dB_c
+ *   grad_theta  float[n_blocks][n_par] = dL/dtheta_c (overwritten)
+ * Arithmetic in fp64, one rounding to fp32.  HARP_ERR_BAD_SCHEDULE if I + A is singular. */
+harp_status_t harp_grad_theta(int32_t b, int64_t n_blocks, const float *theta, const float *mixer,
+                              const float *grad_blocks, float *grad_theta);
+
 /* harp_plan_create with every stage's blocks rebuilt by harp_blocks_from_theta.  theta, theta_q,
  * scales, mixers are HOST arrays of n_stages pointers (theta or theta_q may be NULL as a whole;
  * mixers may be NULL if every radix is a power of two). */

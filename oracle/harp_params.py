@@ -5,6 +5,7 @@
                          b = 2 (Eq. 10) and the Cayley map Q = (I + A)^{-1} (I - A) of a
                          skew-symmetric A for b > 2 (Eq. 11); A is given by its strict upper
                          triangle (row-major, i < j), A_ji = -A_ij.
+* grad_theta           : chain rule from dL/dB back to theta through Eq. 9-11.
 * dequantize_theta     : int8 storage (appendix "Int8 storage of HARP parameters"):
                          a ~ s * q with one scale per block.
 * quantize_theta       : s = max|a| / 127, q = round(a / s).
@@ -69,6 +70,32 @@ def blocks_from_theta(b: int, theta: np.ndarray, mixer: Optional[np.ndarray] = N
     g = sylvester(b) if mixer is None else np.asarray(mixer, dtype=np.float64)
     theta = np.asarray(theta, dtype=np.float64).reshape(-1, n_params(b))
     return np.stack([rotation(b, th) @ g for th in theta])
+
+
+def grad_theta(b: int, theta: np.ndarray, grad_blocks: np.ndarray, mixer: Optional[np.ndarray] = None) -> np.ndarray:
+    """dL/dtheta[n_blocks, n_params(b)] from dL/dB[n_blocks, b, b] for B = Q(theta) G_b (Eq. 9-11).
+
+    D = dL/dQ = (dL/dB) G^T.  Givens (Eq. 10): dL/dtheta = <D, dQ/dtheta>.  Cayley (Eq. 11):
+    differentiating (I + A) Q = I - A gives dQ = -(I + A)^{-1} dA (Q + I), so
+    dL/dA = -(I + A)^{-T} D (Q + I)^T, and the entry of the pair i < j is (dL/dA)_ij - (dL/dA)_ji
+    because A_ji = -A_ij."""
+    g = sylvester(b) if mixer is None else np.asarray(mixer, dtype=np.float64)
+    theta = np.asarray(theta, dtype=np.float64).reshape(-1, n_params(b))
+    gb = np.asarray(grad_blocks, dtype=np.float64).reshape(-1, b, b)
+    out = np.empty_like(theta)
+    eye = np.eye(b)
+    iu = np.triu_indices(b, 1)
+    for c, th in enumerate(theta):
+        dq = gb[c] @ g.T
+        if b == 2:
+            cs, sn = np.cos(th[0]), np.sin(th[0])
+            out[c, 0] = np.sum(dq * np.array([[-sn, -cs], [cs, -sn]]))
+            continue
+        a = skew_from_upper(b, th)
+        q = np.linalg.solve(eye + a, eye - a)
+        da = -np.linalg.solve((eye + a).T, dq) @ (q + eye).T
+        out[c] = (da - da.T)[iu]
+    return out
 
 
 def quantize_theta(theta: np.ndarray):

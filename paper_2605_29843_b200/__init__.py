@@ -45,6 +45,8 @@ def lib() -> ctypes.CDLL:
         L.harp_theta_params_per_block.argtypes = [i32]
         L.harp_blocks_from_theta.restype = ctypes.c_int
         L.harp_blocks_from_theta.argtypes = [i32, i64, vp, vp, vp, vp, vp]
+        L.harp_grad_theta.restype = ctypes.c_int
+        L.harp_grad_theta.argtypes = [i32, i64, vp, vp, vp, vp]
         L.harp_plan_create_from_theta.restype = ctypes.c_int
         L.harp_plan_create_from_theta.argtypes = [ctypes.POINTER(vp), i64, i32, vp, vp, vp, vp, vp, vp, vp]
         L.harp_plan_create_kronecker.restype = ctypes.c_int
@@ -168,6 +170,22 @@ def harp_blocks_from_theta(b: int, theta=None, theta_q=None, scales=None, mixer=
                                       None if mx is None else mx.ctypes.data, out.ctypes.data)
     if st != HARP_OK:
         raise HarpError(st, "harp_blocks_from_theta")
+    return out
+
+
+def harp_grad_theta(b: int, theta, grad_blocks, mixer=None) -> np.ndarray:
+    """Host-only: dL/dtheta[n_blocks, n_par] (float32) from dL/dB[n_blocks, b, b]."""
+    npar = harp_theta_params_per_block(b)
+    th = np.ascontiguousarray(theta, dtype=np.float32).reshape(-1, npar)
+    gb = np.ascontiguousarray(grad_blocks, dtype=np.float32).reshape(-1, b, b)
+    if gb.shape[0] != th.shape[0]:
+        raise ValueError("theta and grad_blocks disagree on the number of blocks")
+    mx = None if mixer is None else np.ascontiguousarray(mixer, dtype=np.float32)
+    out = np.empty_like(th)
+    st = lib().harp_grad_theta(int(b), th.shape[0], th.ctypes.data, None if mx is None else mx.ctypes.data,
+                               gb.ctypes.data, out.ctypes.data)
+    if st != HARP_OK:
+        raise HarpError(st, "harp_grad_theta")
     return out
 
 

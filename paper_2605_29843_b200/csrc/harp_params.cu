@@ -124,6 +124,65 @@ extern "C" harp_status_t harp_blocks_from_theta(int32_t b, int64_t n_blocks, con
     return HARP_OK;
 }
 
+// Chain rule from the block kernels back to the stored parameters.  K = Q G, so D = dL/dQ = (dL/dK) G^T.
+// Givens: dL/dtheta = <D, dQ/dtheta>.  Cayley: with M = (I + A)^{-1} = (Q + I)/2, a change dA moves Q
+// by -M dA (Q + I), hence dL/dA = -(1/2) (Q + I)^T D (Q + I)^T, and the parameter of the pair i < j
+// (A_ij = a, A_ji = -a) collects (dL/dA)_ij - (dL/dA)_ji.
+extern "C" harp_status_t harp_grad_theta(int32_t b, int64_t n_blocks, const float *theta, const float *mixer,
+                                         const float *grad_blocks, float *grad_theta) {
+    if (!theta || !grad_blocks || !grad_theta) return HARP_ERR_NULL;
+    if (b < 2 || b > 256 || n_blocks < 0) return HARP_ERR_BAD_SCHEDULE;
+    if (!mixer && !is_pow2(b)) return HARP_ERR_NULL;
+    const int np = harp_theta_params_per_block(b);
+    const size_t bb = (size_t)b * b;
+    std::vector<double> g, q, th((size_t)np), dq, p, tmp;
+    try {
+        if (mixer) {
+            g.resize(bb);
+            for (size_t i = 0; i < bb; ++i) g[i] = mixer[i];
+        } else {
+            sylvester(b, g);
+        }
+        q.resize(bb); dq.resize(bb); p.resize(bb); tmp.resize(bb);
+    } catch (const std::bad_alloc &) {
+        return HARP_ERR_ALLOC;
+    }
+    for (int64_t c = 0; c < n_blocks; ++c) {
+        const float *gk = grad_blocks + c * (int64_t)bb;
+        for (int i = 0; i < b; ++i)                       // D = (dL/dK) G^T
+            for (int k = 0; k < b; ++k) {
+                double acc = 0.0;
+                for (int j = 0; j < b; ++j) acc += (double)gk[i * b + j] * g[(size_t)k * b + j];
+                dq[(size_t)i * b + k] = acc;
+            }
+        for (int k = 0; k < np; ++k) th[(size_t)k] = theta[c * np + k];
+        float *out = grad_theta + c * np;
+        if (b == 2) {
+            const double cs = std::cos(th[0]), sn = std::sin(th[0]);
+            out[0] = (float)(-sn * dq[0] - cs * dq[1] + cs * dq[2] - sn * dq[3]);
+            continue;
+        }
+        if (!cayley(b, th.data(), q)) return HARP_ERR_BAD_SCHEDULE;
+        for (int i = 0; i < b; ++i)                       // P = Q + I
+            for (int j = 0; j < b; ++j) p[(size_t)i * b + j] = q[(size_t)i * b + j] + (i == j ? 1.0 : 0.0);
+        for (int i = 0; i < b; ++i)                       // tmp = P^T D
+            for (int j = 0; j < b; ++j) {
+                double acc = 0.0;
+                for (int k = 0; k < b; ++k) acc += p[(size_t)k * b + i] * dq[(size_t)k * b + j];
+                tmp[(size_t)i * b + j] = acc;
+            }
+        auto ga = [&](int i, int j) {                     // (dL/dA)_ij = -(1/2) (tmp P^T)_ij
+            double acc = 0.0;
+            for (int k = 0; k < b; ++k) acc += tmp[(size_t)i * b + k] * p[(size_t)j * b + k];
+            return -0.5 * acc;
+        };
+        int k = 0;
+        for (int i = 0; i < b; ++i)
+            for (int j = i + 1; j < b; ++j, ++k) out[k] = (float)(ga(i, j) - ga(j, i));
+    }
+    return HARP_OK;
+}
+
 extern "C" harp_status_t harp_plan_create_from_theta(harp_plan_t **out, int64_t d, int32_t n_stages, const int32_t *radices,
                                                      const int32_t *perm, const int8_t *signs, const float *const *theta,
                                                      const int8_t *const *theta_q, const float *const *scales,

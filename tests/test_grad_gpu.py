@@ -6,6 +6,7 @@ import torch
 
 import paper_2605_29843_b200 as harp
 from oracle import harp_oracle as orc
+from oracle import harp_params as prm
 from paper_2605_29843_b200 import workloads as wl
 from harp_testlib import host_rows, promote, to_device
 
@@ -106,3 +107,38 @@ def test_euler_identity_at_full_dimension():
         off += k.numel()
         assert got == pytest.approx(L, rel=2e-4), t
     assert off == grad.numel()
+
+
+def test_parameter_gradient_of_a_plan_built_from_theta():
+    """One parameter step's worth of Algorithm 3 without the quantizer: plan from theta, L = sum(y * G)
+    with y from harp_apply, dL/dK on the GPU, dL/dtheta on the host; compared with central
+    differences of the fp64 oracle (theta -> blocks -> forward) on sampled parameters."""
+    radices, d = (4, 2, 8), 64
+    rng = np.random.default_rng(70)
+    theta = [rng.normal(0, 0.3, (d // b, prm.n_params(b))).astype(np.float32) for b in radices]
+    perm = rng.permutation(d).astype(np.int32)
+    signs = rng.choice(np.array([-1, 1], dtype=np.int8), d)
+    plan = harp.harp_plan_create_from_theta(d, radices, perm=perm, signs=signs, theta=theta)
+    xh = host_rows(rng.standard_normal((50, d)), "f32")
+    gh = host_rows(rng.standard_normal((50, d)), "f32")
+    grad, _, _ = _gpu_grad(plan, xh, gh, "f32")
+
+    def loss(th_list):
+        blocks = [prm.blocks_from_theta(b, th.astype(np.float64)) for b, th in zip(radices, th_list)]
+        op = orc.OraclePlan(d, radices, perm, signs, [np.float32(k) for k in blocks])
+        return float(np.sum(orc.forward(op, promote(xh, "f32")) * promote(gh, "f32")))
+
+    off = 0
+    for t, b in enumerate(radices):
+        n = d * b
+        g_theta = harp.harp_grad_theta(b, theta[t], grad[off:off + n].reshape(d // b, b, b))
+        off += n
+        for c, k in [(0, 0), (d // b - 1, prm.n_params(b) - 1), (3, 0)]:
+            h = 1e-3
+            tp = [a.astype(np.float64) for a in theta]
+            tm = [a.astype(np.float64) for a in theta]
+            tp[t][c, k] += h
+            tm[t][c, k] -= h
+            # the loss is smooth; blocks are rounded to fp32 inside loss(), hence the loose step and bound
+            fd = (loss(tp) - loss(tm)) / (2 * h)
+            assert abs(g_theta[c, k] - fd) <= 2e-3 * max(1.0, abs(fd)), (t, c, k, g_theta[c, k], fd)

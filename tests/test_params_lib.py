@@ -45,6 +45,24 @@ def test_blocks_from_theta_match_oracle(b):
     assert np.max(np.abs(np.swapaxes(got, 1, 2).astype(np.float64) @ got - np.eye(b))) < 2e-6
 
 
+@pytest.mark.parametrize("b", [2, 3, 4, 5, 7, 8, 16, 43])
+def test_grad_theta_matches_oracle(b):
+    rng = np.random.default_rng(60 + b)
+    npar = harp.harp_theta_params_per_block(b)
+    theta = rng.normal(0, 0.3, (7, npar)).astype(np.float32)
+    gb = rng.standard_normal((7, b, b)).astype(np.float32)
+    mixer = None if (b & (b - 1)) == 0 else np.linalg.qr(rng.standard_normal((b, b)))[0].astype(np.float32)
+    got = harp.harp_grad_theta(b, theta, gb, mixer)
+    want = prm.grad_theta(b, theta.astype(np.float64), gb.astype(np.float64), None if mixer is None else mixer.astype(np.float64))
+    assert got.shape == want.shape == (7, npar)
+    assert np.max(np.abs(got - want)) <= 1e-6 * max(1.0, np.max(np.abs(want)))
+    L = harp.lib()
+    assert L.harp_grad_theta(b, 7, None, None, gb.ctypes.data, got.ctypes.data) == 1
+    assert L.harp_grad_theta(1, 7, theta.ctypes.data, None, gb.ctypes.data, got.ctypes.data) == 3
+    if mixer is not None:                                     # no default mixer for this radix
+        assert L.harp_grad_theta(b, 7, theta.ctypes.data, None, gb.ctypes.data, got.ctypes.data) == 1
+
+
 def test_int8_parameters():
     rng = np.random.default_rng(5)
     b = 8

@@ -68,6 +68,47 @@ def test_cayley_closed_form_and_properties():
         assert np.allclose(q, scipy.linalg.inv(np.eye(b) + A) @ (np.eye(b) - A), atol=1e-13)
 
 
+@pytest.mark.parametrize("b", [2, 3, 4, 7, 8, 16])
+def test_grad_theta_against_finite_differences(b):
+    """L(theta) = <W, B(theta)> with a fixed W: central differences of the block reconstruction pin
+    the chain rule (signs, transposes, which triangle entry belongs to which parameter)."""
+    rng = np.random.default_rng(40 + b)
+    npar = prm.n_params(b)
+    theta = rng.normal(0, 0.4, (3, npar))
+    w = rng.standard_normal((3, b, b))
+    mixer = None if (b & (b - 1)) == 0 else np.linalg.qr(rng.standard_normal((b, b)))[0]
+    got = prm.grad_theta(b, theta, w, mixer)
+    h = 1e-6
+    for c in range(3):
+        for k in range(npar):
+            tp, tm = theta.copy(), theta.copy()
+            tp[c, k] += h
+            tm[c, k] -= h
+            fd = (np.sum(w * prm.blocks_from_theta(b, tp, mixer)) - np.sum(w * prm.blocks_from_theta(b, tm, mixer))) / (2 * h)
+            assert abs(got[c, k] - fd) <= 1e-7 * max(1.0, abs(fd)), (c, k)
+
+
+def test_grad_theta_closed_forms():
+    rng = np.random.default_rng(50)
+    # theta = 0, identity mixer: Q = I, dQ = -2 dA, so dL/da_ij = -2 (W_ij - W_ji)
+    for b in (3, 4, 6):
+        w = rng.standard_normal((1, b, b))
+        got = prm.grad_theta(b, np.zeros((1, prm.n_params(b))), w, np.eye(b))[0]
+        want = (-2.0 * (w[0] - w[0].T))[np.triu_indices(b, 1)]
+        assert np.allclose(got, want, atol=1e-14)
+    # Givens, identity mixer: L = W00 c - W01 s + W10 s + W11 c
+    th, w = 0.3, rng.standard_normal((1, 2, 2))
+    got = prm.grad_theta(2, np.array([[th]]), w, np.eye(2))[0, 0]
+    assert np.isclose(got, -(w[0, 0, 0] + w[0, 1, 1]) * np.sin(th) + (w[0, 1, 0] - w[0, 0, 1]) * np.cos(th))
+    # a loss that depends on Q only through Q^T Q (= I for every theta) has zero gradient:
+    # L = ||B||_F^2 / 2 with an orthogonal mixer, dL/dB = B
+    for b in (2, 5, 8):
+        theta = rng.normal(0, 0.5, (4, prm.n_params(b)))
+        g = np.linalg.qr(rng.standard_normal((b, b)))[0]
+        blocks = prm.blocks_from_theta(b, theta, g)
+        assert np.max(np.abs(prm.grad_theta(b, theta, blocks, g))) < 1e-13
+
+
 def test_int8_storage_error_bound():
     rng = np.random.default_rng(2)
     theta = rng.normal(0, 0.2, (50, 28))
