@@ -115,6 +115,25 @@ extern "C" harp_status_t harp_plan_create(harp_plan_t **out, int64_t d, int32_t 
     if (st == HARP_OK &&
         cudaMemcpy(p->d_blocks, p->h_blocks.data(), sizeof(float) * (size_t)off, cudaMemcpyHostToDevice) != cudaSuccess)
         st = HARP_ERR_CUDA;
+    if (st == HARP_OK) {         // element-major copy (neighbouring blocks' entries side by side), for the gradient kernels
+        std::vector<float> em;
+        try {
+            em.resize((size_t)off);
+        } catch (const std::bad_alloc &) {
+            st = HARP_ERR_ALLOC;
+        }
+        for (int t = 0; st == HARP_OK && t < p->st.m; ++t) {
+            const int64_t bb = (int64_t)p->st.b[t] * p->st.b[t], nblk = d / p->st.b[t];
+            const float *src = p->h_blocks.data() + p->st.off[t];
+            float *dst = em.data() + p->st.off[t];
+            for (int64_t c = 0; c < nblk; ++c)
+                for (int64_t k = 0; k < bb; ++k) dst[k * nblk + c] = src[c * bb + k];
+        }
+        if (st == HARP_OK && cudaMalloc(&p->d_blocks_em, sizeof(float) * (size_t)off) != cudaSuccess) st = HARP_ERR_ALLOC;
+        if (st == HARP_OK &&
+            cudaMemcpy(p->d_blocks_em, em.data(), sizeof(float) * (size_t)off, cudaMemcpyHostToDevice) != cudaSuccess)
+            st = HARP_ERR_CUDA;
+    }
     if (st == HARP_OK && p->d_perm &&
         cudaMemcpy(p->d_perm, p->h_perm.data(), sizeof(int32_t) * (size_t)d, cudaMemcpyHostToDevice) != cudaSuccess)
         st = HARP_ERR_CUDA;
@@ -155,6 +174,7 @@ extern "C" void harp_plan_destroy(harp_plan_t *p) {
             if (p->stage_buf[i]) cudaFree(p->stage_buf[i]);
         }
         if (p->d_blocks) cudaFree(p->d_blocks);
+        if (p->d_blocks_em) cudaFree(p->d_blocks_em);
         if (p->d_fused_blocks) cudaFree(p->d_fused_blocks);
         if (p->d_bo_blocks) cudaFree(p->d_bo_blocks);
         if (p->d_perm) cudaFree(p->d_perm);

@@ -226,20 +226,24 @@ load_kernel(const T *__restrict__ x, const T *__restrict__ gy, int64_t rows, int
     }
 }
 
-// one stage on a chunk: out[r][base + j s] = sum_i in[r][base + i s] * K[c][i][j]   (transpose: K[c][j][i])
+// one stage on a chunk: out[r][base + j s] = sum_i in[r][base + i s] * K[c][i][j]   (transpose: K[c][j][i]).
+// Neighbouring lanes hold neighbouring positions: inside one block when s is small, in neighbouring
+// blocks otherwise -- so K is read block-major (entry k of block c at c b^2 + k) for s < 8 and
+// element-major (at k D + c) from s = 8 on; kc_step / kk_step are the two strides of that choice.
 __global__ void __launch_bounds__(kThreads)
 stage_kernel(const float *__restrict__ in, float *__restrict__ out, int64_t rows, int64_t d, int b, int64_t s,
-             const float *__restrict__ K, int transpose) {
+             const float *__restrict__ K, int64_t kc_step, int64_t kk_step, int transpose) {
     const int64_t total = rows * d;
     for (int64_t e = (int64_t)blockIdx.x * kThreads + threadIdx.x; e < total; e += (int64_t)gridDim.x * kThreads) {
         const int64_t r = e / d, pos = e - r * d;
         const int64_t alpha = pos / (b * s), rem = pos - alpha * b * s;
         const int64_t j = rem / s, beta = rem - j * s;
         const int64_t base = alpha * b * s + beta;
-        const float *Kc = K + (alpha * s + beta) * b * b;
+        const float *Kc = K + (alpha * s + beta) * kc_step;
         const float *row = in + r * d + base;
         float acc = 0.f;
-        for (int i = 0; i < b; ++i) acc = fmaf(row[(int64_t)i * s], Kc[transpose ? j * b + i : (int64_t)i * b + j], acc);
+        for (int i = 0; i < b; ++i)
+            acc = fmaf(row[(int64_t)i * s], Kc[(transpose ? j * b + i : (int64_t)i * b + j) * kk_step], acc);
         out[e] = acc;
     }
 }
@@ -247,17 +251,22 @@ stage_kernel(const float *__restrict__ in, float *__restrict__ out, int64_t rows
 // grad[c][i][j] (+)= sum_r v[r][base_c + i s] * g[r][base_c + j s].  A CTA owns 32 neighbouring
 // entries (one per lane); its eight warps take the rows r = w, w + 8, ... and their partial sums
 // are added in a fixed order, so the result does not depend on scheduling.
+// The 32 entries are neighbours within a block for s < 8 and the same entry of 32 neighbouring
+// blocks from s = 8 on (by_block = 0), so that the lanes read neighbouring coordinates either way.
 __global__ void __launch_bounds__(kThreads)
 outer_kernel(const float *__restrict__ v, const float *__restrict__ g, int64_t rows, int64_t d, int b, int64_t s,
-             float *__restrict__ grad, int accumulate) {
+             float *__restrict__ grad, int accumulate, int by_block) {
     __shared__ double part[kThreads / 32][32];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int64_t total = d * b;                       // (d / b) blocks of b*b entries
+    const int64_t nblk = d / b;
     for (int64_t e0 = (int64_t)blockIdx.x * 32; e0 < total; e0 += (int64_t)gridDim.x * 32) {
-        const int64_t e = e0 + lane;
+        const int64_t q = e0 + lane;
+        int64_t e = q;
         double acc = 0.0;
-        if (e < total) {
-            const int64_t c = e / (b * b), ij = e - c * b * b;
+        if (q < total) {
+            const int64_t c = by_block ? q / (b * b) : q % nblk, ij = by_block ? q - c * b * b : q / nblk;
+            e = c * b * b + ij;
             const int64_t i = ij / b, j = ij - i * b;
             const int64_t alpha = c / s, beta = c - alpha * s;
             const int64_t base = alpha * b * s + beta;
@@ -266,7 +275,7 @@ outer_kernel(const float *__restrict__ v, const float *__restrict__ g, int64_t r
         }
         part[w][lane] = acc;
         __syncthreads();
-        if (w == 0 && e < total) {
+        if (w == 0 && q < total) {
             double sum = part[0][lane];
             for (int k = 1; k < kThreads / 32; ++k) sum += part[k][lane];
             grad[e] = accumulate ? grad[e] + (float)sum : (float)sum;
@@ -364,8 +373,11 @@ extern "C" harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x
         for (int t = 0; t + 1 < m; ++t, ++launches) {
             const int b = plan->st.b[t];
             const float *K = plan->d_blocks + plan->st.off[t];
+            const bool em = plan->st.s[t] >= 8;             // see stage_kernel
             if (owner_radix(b)) launch_fwd_owner(b, scratch + t * plane, scratch + (t + 1) * plane, rows, d, plan->st.s[t], K, st);
-            else stage_kernel<<<grid, kThreads, 0, st>>>(scratch + t * plane, scratch + (t + 1) * plane, rows, d, b, plan->st.s[t], K, 0);
+            else stage_kernel<<<grid, kThreads, 0, st>>>(scratch + t * plane, scratch + (t + 1) * plane, rows, d, b, plan->st.s[t],
+                                                         em ? plan->d_blocks_em + plan->st.off[t] : K, em ? 1 : (int64_t)b * b,
+                                                         em ? d / b : 1, 0);
         }
         // backward: entry sums, and the gradient state one stage back
         float *g_cur = ga, *g_nxt = gb;
@@ -380,9 +392,12 @@ extern "C" harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x
                                                                            grad + plan->st.off[t], acc);
                 launches += 2;
             } else {
-                outer_kernel<<<(unsigned)std::min<int64_t>((d * b + 31) / 32, 148 * 64), kThreads, 0, st>>>(scratch + t * plane, g_cur, rows,
-                                                                                                         d, b, s, grad + plan->st.off[t], acc);
-                if (t > 0) stage_kernel<<<grid, kThreads, 0, st>>>(g_cur, g_nxt, rows, d, b, s, K, 1);
+                const bool em = s >= 8;
+                outer_kernel<<<(unsigned)std::min<int64_t>((d * b + 31) / 32, 148 * 64), kThreads, 0, st>>>(
+                    scratch + t * plane, g_cur, rows, d, b, s, grad + plan->st.off[t], acc, em ? 0 : 1);
+                if (t > 0)
+                    stage_kernel<<<grid, kThreads, 0, st>>>(g_cur, g_nxt, rows, d, b, s, em ? plan->d_blocks_em + plan->st.off[t] : K,
+                                                            em ? 1 : (int64_t)b * b, em ? d / b : 1, 1);
                 launches += t > 0 ? 2 : 1;
             }
             if (t > 0) std::swap(g_cur, g_nxt);

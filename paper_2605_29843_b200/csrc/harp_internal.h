@@ -30,6 +30,7 @@ struct harp_plan {
     StageTable st{};
     int64_t n_params = 0;
     float *d_blocks = nullptr;        // [sum_t d*b_t] fp32, stage after stage
+    float *d_blocks_em = nullptr;     // the same stages element-major: entry k of block c of stage t at off[t] + k*D_t + c
     // the same map with runs of small-radix stages fused into dense blocks of size <= 4 (fewer
     // stages for the CUDA-core kernel); fused.m == 0 if nothing could be fused
     StageTable fused{};
