@@ -10,7 +10,7 @@
 // scratch (fp32) and the gradient state is walked back stage by stage.  Every sum over rows is
 // taken in fp64 in a fixed order -- no atomics, so the result does not depend on scheduling.
 //
-// Stages of radix 2, 4 and 8 run in "block owner" kernels: a thread owns one block c of the stage,
+// Stages of radix 2 to 8 run in "block owner" kernels: a thread owns one block c of the stage,
 // keeps K_t[c] in registers and walks the rows of its slice of the chunk, so neighbouring lanes
 // read neighbouring coordinates (or one vector when s_t = 1) and K is read once.  The backward
 // kernel of such a stage does both jobs in one sweep over v_t and g_{t+1}: it writes g_t and adds
@@ -34,7 +34,7 @@ constexpr int kBwdSliceRows = 16;  //                      rows per CTA (one set
 constexpr int kRowBatch = 4;       //                      rows whose loads are issued together
 
 template <int B> __device__ __forceinline__ void load_block(const float *p, int64_t s, float (&v)[B]) {
-    if (s == 1) {
+    if (s == 1 && (B == 2 || B % 4 == 0)) {
         if constexpr (B == 2) {
             const float2 a = *reinterpret_cast<const float2 *>(p);
             v[0] = a.x; v[1] = a.y;
@@ -52,7 +52,7 @@ template <int B> __device__ __forceinline__ void load_block(const float *p, int6
 }
 
 template <int B> __device__ __forceinline__ void store_block(float *p, int64_t s, const float (&v)[B]) {
-    if (s == 1) {
+    if (s == 1 && (B == 2 || B % 4 == 0)) {
         if constexpr (B == 2) {
             *reinterpret_cast<float2 *>(p) = make_float2(v[0], v[1]);
         } else {
@@ -120,7 +120,7 @@ bwd_owner_kernel(const float *__restrict__ v, const float *__restrict__ g, float
             acc[i][j] = 0.0;
         }
     const int64_t alpha = c / s, base = alpha * B * s + (c - alpha * s);
-    constexpr int U = B == 8 ? 2 : kRowBatch;         // radix 8 already fills the register file
+    constexpr int U = B >= 7 ? 2 : kRowBatch;         // radices 7 and 8 already fill the register file
     const int64_t r0 = (int64_t)blockIdx.y * kBwdSliceRows, r1 = min(rows, r0 + kBwdSliceRows);
     for (int64_t r = r0; r < r1; r += U) {
         float vv[U][B], gg[U][B];
@@ -288,7 +288,7 @@ unsigned grid_for(int64_t work) {
     return (unsigned)std::max<int64_t>(1, std::min<int64_t>((work + kThreads - 1) / kThreads, 148 * 16));
 }
 
-bool owner_radix(int b) { return b == 2 || b == 4 || b == 8; }
+bool owner_radix(int b) { return b >= 2 && b <= 8; }
 
 dim3 owner_grid(int64_t d, int b, int64_t rows, int slice_rows) {
     return dim3((unsigned)((d / b + kOwnThreads - 1) / kOwnThreads), (unsigned)((rows + slice_rows - 1) / slice_rows));
@@ -296,17 +296,29 @@ dim3 owner_grid(int64_t d, int b, int64_t rows, int slice_rows) {
 
 void launch_fwd_owner(int b, const float *in, float *out, int64_t rows, int64_t d, int64_t s, const float *K, cudaStream_t st) {
     const dim3 grid = owner_grid(d, b, rows, kFwdSliceRows);
-    if (b == 2) fwd_owner_kernel<2><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K);
-    else if (b == 4) fwd_owner_kernel<4><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K);
-    else fwd_owner_kernel<8><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K);
+    switch (b) {
+        case 2: fwd_owner_kernel<2><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K); break;
+        case 3: fwd_owner_kernel<3><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K); break;
+        case 4: fwd_owner_kernel<4><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K); break;
+        case 5: fwd_owner_kernel<5><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K); break;
+        case 6: fwd_owner_kernel<6><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K); break;
+        case 7: fwd_owner_kernel<7><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K); break;
+        default: fwd_owner_kernel<8><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K); break;
+    }
 }
 
 void launch_bwd_owner(int b, const float *v, const float *g, float *g_out, int64_t rows, int64_t d, int64_t s, const float *K,
                       double *part, cudaStream_t st) {
     const dim3 grid = owner_grid(d, b, rows, kBwdSliceRows);
-    if (b == 2) bwd_owner_kernel<2><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part);
-    else if (b == 4) bwd_owner_kernel<4><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part);
-    else bwd_owner_kernel<8><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part);
+    switch (b) {
+        case 2: bwd_owner_kernel<2><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part); break;
+        case 3: bwd_owner_kernel<3><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part); break;
+        case 4: bwd_owner_kernel<4><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part); break;
+        case 5: bwd_owner_kernel<5><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part); break;
+        case 6: bwd_owner_kernel<6><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part); break;
+        case 7: bwd_owner_kernel<7><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part); break;
+        default: bwd_owner_kernel<8><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part); break;
+    }
 }
 
 template <typename T>
