@@ -157,6 +157,84 @@ bwd_owner_kernel(const float *__restrict__ v, const float *__restrict__ g, float
         for (int j = 0; j < B; ++j) dst[(int64_t)(i * B + j) * nblk] = acc[i][j];
 }
 
+// Radix 16: a block kernel does not fit one thread's registers, so a thread owns block c and four
+// of its sixteen outputs (forward: columns j0..j0+3 of K[c]; backward: rows i0..i0+3, i.e. the
+// transposed product), with the four threads of a block in the same CTA so that they share the
+// sixteen inputs through L1.
+constexpr int kTileRows16 = 32;    // rows per CTA of the radix-16 kernels (one set of partial sums)
+
+__global__ void __launch_bounds__(128)
+stage16_kernel(const float *__restrict__ in, float *__restrict__ out, int64_t rows, int64_t d, int64_t s,
+               const float *__restrict__ K, int transpose) {
+    const int64_t c = (int64_t)blockIdx.x * 32 + (threadIdx.x & 31);
+    const int t0 = 4 * (threadIdx.x >> 5);
+    if (c >= d / 16) return;
+    float k[16][4];
+#pragma unroll
+    for (int q = 0; q < 16; ++q)
+#pragma unroll
+        for (int t = 0; t < 4; ++t) k[q][t] = K[c * 256 + (transpose ? (t0 + t) * 16 + q : q * 16 + t0 + t)];
+    const int64_t alpha = c / s, base = alpha * 16 * s + (c - alpha * s);
+    const int64_t r0 = (int64_t)blockIdx.y * kFwdSliceRows, r1 = min(rows, r0 + kFwdSliceRows);
+#pragma unroll 2
+    for (int64_t r = r0; r < r1; ++r) {
+        float v[16];
+        load_block<16>(in + r * d + base, s, v);
+        float o[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int q = 0; q < 16; ++q)
+#pragma unroll
+            for (int t = 0; t < 4; ++t) o[t] = fmaf(v[q], k[q][t], o[t]);
+        float *dst = out + r * d + base + (int64_t)t0 * s;
+        if (s == 1) {
+            *reinterpret_cast<float4 *>(dst) = make_float4(o[0], o[1], o[2], o[3]);
+        } else {
+#pragma unroll
+            for (int t = 0; t < 4; ++t) dst[(int64_t)t * s] = o[t];
+        }
+    }
+}
+
+// part[slice][i 16 + j][c] = sum over the slice's rows of v[base_c + i s] g[base_c + j s]; a thread
+// owns block c and a 4 x 4 tile of (i, j); the sixteen tiles of a block sit in the same CTA.
+__global__ void __launch_bounds__(512)
+outer16_kernel(const float *__restrict__ v, const float *__restrict__ g, int64_t rows, int64_t d, int64_t s,
+               double *__restrict__ part) {
+    const int64_t nblk = d / 16;
+    const int64_t c = (int64_t)blockIdx.x * 32 + (threadIdx.x & 31);
+    const int tile = threadIdx.x >> 5, i0 = 4 * (tile >> 2), j0 = 4 * (tile & 3);
+    if (c >= nblk) return;
+    double acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+    const int64_t alpha = c / s, base = alpha * 16 * s + (c - alpha * s);
+    const int64_t r0 = (int64_t)blockIdx.y * kTileRows16, r1 = min(rows, r0 + kTileRows16);
+    for (int64_t r = r0; r < r1; r += 2) {
+        float vv[2][4], gg[2][4];
+#pragma unroll
+        for (int u = 0; u < 2; ++u)
+            if (r + u < r1) {
+                load_block<4>(v + (r + u) * d + base + (int64_t)i0 * s, s, vv[u]);
+                load_block<4>(g + (r + u) * d + base + (int64_t)j0 * s, s, gg[u]);
+            }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            if (r + u >= r1) break;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] += (double)vv[u][i] * (double)gg[u][j];
+        }
+    }
+    double *dst = part + (int64_t)blockIdx.y * 256 * nblk + c;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) dst[(int64_t)((i0 + i) * 16 + j0 + j) * nblk] = acc[i][j];
+}
+
 // grad[c][i][j] (+)= sum over slices of part[slice][i b + j][c].  A CTA owns 32 neighbouring
 // entries (one per lane); warp w adds the slices w, w + 8, ... and the eight sums are added in
 // the order of w, so the result does not depend on scheduling.
@@ -290,6 +368,10 @@ unsigned grid_for(int64_t work) {
 
 bool owner_radix(int b) { return b >= 2 && b <= 8; }
 
+dim3 owner_grid16(int64_t d, int64_t rows, int slice_rows) {
+    return dim3((unsigned)((d / 16 + 31) / 32), (unsigned)((rows + slice_rows - 1) / slice_rows));
+}
+
 dim3 owner_grid(int64_t d, int b, int64_t rows, int slice_rows) {
     return dim3((unsigned)((d / b + kOwnThreads - 1) / kOwnThreads), (unsigned)((rows + slice_rows - 1) / slice_rows));
 }
@@ -354,14 +436,16 @@ extern "C" harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x
         return HARP_OK;
     }
     // chunk of rows whose m forward states, two gradient states and the per-slice sums of the
-    // block-owner stages (at most one state: 8 bytes x d b / 16 per row, b <= 8) fit ~256 MB
+    // block-owner stages (at most one state: 8 bytes x d b / 16 per row for b <= 8, d b / 32 for b = 16) fit ~256 MB
     const int64_t per_row = (int64_t)(m + 3) * d * (int64_t)sizeof(float);
     const int64_t chunk = std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(n_rows, 1 << 18), (256ll << 20) / per_row));
-    int max_owner_b = 0;
-    for (int t = 0; t < m; ++t)
-        if (owner_radix(plan->st.b[t])) max_owner_b = std::max(max_owner_b, plan->st.b[t]);
+    int64_t part_bytes = 0;                          // per-slice sums of the stage that needs most
+    for (int t = 0; t < m; ++t) {
+        const int b = plan->st.b[t];
+        const int slice = owner_radix(b) ? kBwdSliceRows : (b == 16 ? kTileRows16 : 0);
+        if (slice) part_bytes = std::max<int64_t>(part_bytes, ((chunk + slice - 1) / slice) * d * b * (int64_t)sizeof(double));
+    }
     const int64_t state_bytes = (int64_t)(m + 2) * chunk * d * (int64_t)sizeof(float);
-    const int64_t part_bytes = ((chunk + kBwdSliceRows - 1) / kBwdSliceRows) * d * max_owner_b * (int64_t)sizeof(double);
     float *scratch = nullptr;
     if (cudaMallocAsync(reinterpret_cast<void **>(&scratch), (size_t)(state_bytes + 256 + part_bytes), st) != cudaSuccess) {
         cudaGetLastError();
@@ -387,6 +471,7 @@ extern "C" harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x
             const float *K = plan->d_blocks + plan->st.off[t];
             const bool em = plan->st.s[t] >= 8;             // see stage_kernel
             if (owner_radix(b)) launch_fwd_owner(b, scratch + t * plane, scratch + (t + 1) * plane, rows, d, plan->st.s[t], K, st);
+            else if (b == 16) stage16_kernel<<<owner_grid16(d, rows, kFwdSliceRows), 128, 0, st>>>(scratch + t * plane, scratch + (t + 1) * plane, rows, d, plan->st.s[t], K, 0);
             else stage_kernel<<<grid, kThreads, 0, st>>>(scratch + t * plane, scratch + (t + 1) * plane, rows, d, b, plan->st.s[t],
                                                          em ? plan->d_blocks_em + plan->st.off[t] : K, em ? 1 : (int64_t)b * b,
                                                          em ? d / b : 1, 0);
@@ -403,6 +488,12 @@ extern "C" harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x
                 reduce_slices_kernel<<<(unsigned)std::min<int64_t>((d * b + 31) / 32, 148 * 16), kThreads, 0, st>>>(part, (rows + kBwdSliceRows - 1) / kBwdSliceRows, d / b, b * b,
                                                                            grad + plan->st.off[t], acc);
                 launches += 2;
+            } else if (b == 16) {
+                outer16_kernel<<<owner_grid16(d, rows, kTileRows16), 512, 0, st>>>(scratch + t * plane, g_cur, rows, d, s, part);
+                reduce_slices_kernel<<<(unsigned)std::min<int64_t>((d * b + 31) / 32, 148 * 16), kThreads, 0, st>>>(
+                    part, (rows + kTileRows16 - 1) / kTileRows16, d / b, b * b, grad + plan->st.off[t], acc);
+                if (t > 0) stage16_kernel<<<owner_grid16(d, rows, kFwdSliceRows), 128, 0, st>>>(g_cur, g_nxt, rows, d, s, K, 1);
+                launches += t > 0 ? 3 : 2;
             } else {
                 const bool em = s >= 8;
                 outer_kernel<<<(unsigned)std::min<int64_t>((d * b + 31) / 32, 148 * 64), kThreads, 0, st>>>(

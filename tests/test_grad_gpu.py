@@ -50,7 +50,7 @@ def test_grad_blocks_matches_the_oracle(dtype, radices, perm):
                           to_device(xh, dtype).cpu().view(torch.int16 if dtype == "bf16" else torch.int32).numpy())
 
 
-@pytest.mark.parametrize("radices", [(8, 4, 2), (2, 8), (4, 4, 4), (6, 7), (5, 3, 7)])
+@pytest.mark.parametrize("radices", [(8, 4, 2), (2, 8), (4, 4, 4), (6, 7), (5, 3, 7), (2, 16), (4, 16, 2), (16, 16)])
 def test_rows_spanning_several_slices(radices):
     """More rows than one thread block of the block-owner kernels walks, with a ragged last slice
     and a ragged last batch; radix 8 both at stride one and strided."""
