@@ -217,7 +217,8 @@ int64_t harp_two_sided_static_capacity_bytes(void);
  *              if accumulate != 0
  * Any schedule is accepted.  Sums over rows are taken in fp64 by one thread per entry (no
  * atomics: the result does not depend on scheduling).  The call allocates and frees scratch
- * on the stream (at most ~256 MB); HARP_ERR_ALLOC if that fails.  Asynchronous on stream. */
+ * on the stream (at most ~256 MB, from a memory pool of the library's own that keeps what it has
+ * been given until the process ends); HARP_ERR_ALLOC if that fails.  Asynchronous on stream. */
 harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x, const void *gy, int64_t n_rows,
                                harp_dtype_t dtype, float *grad, int accumulate, void *stream);
 

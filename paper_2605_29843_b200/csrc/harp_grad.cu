@@ -17,12 +17,40 @@
 // v_t[i] g_{t+1}[j] into its B x B fp64 accumulators; the per-slice sums are then added slice by
 // slice.  Other radices use the plain one-thread-per-element kernels below them.
 #include <algorithm>
+#include <map>
+#include <mutex>
 
 #include "harp_internal.h"
 
 namespace {
 
 constexpr int kThreads = 256;
+
+// The kernels of one call form a chain, each reading what the one before wrote, and most last
+// 5-30 us; they are launched with the programmatic stream-serialisation attribute so that the
+// launch of the next one overlaps the tail of the current one.  Each kernel calls
+// prior_kernel_done() before it touches anything a kernel before it wrote (griddepcontrol.wait
+// returns when that kernel has completed and its writes are visible), and only then lets the
+// kernel after it start, so at most one later kernel is resident early.
+__device__ __forceinline__ void prior_kernel_done() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+void launch_dep(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);     // errors are read with cudaGetLastError by the caller
+}
 
 template <typename T> __device__ __forceinline__ float to_f32(T v);
 template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
@@ -78,6 +106,7 @@ fwd_owner_kernel(const float *__restrict__ in, float *__restrict__ out, int64_t 
     for (int i = 0; i < B; ++i)
 #pragma unroll
         for (int j = 0; j < B; ++j) k[i][j] = K[c * (B * B) + i * B + j];
+    prior_kernel_done();
     const int64_t alpha = c / s, base = alpha * B * s + (c - alpha * s);
     const int64_t r0 = (int64_t)blockIdx.y * kFwdSliceRows, r1 = min(rows, r0 + kFwdSliceRows);
     for (int64_t r = r0; r < r1; r += kRowBatch) {
@@ -119,6 +148,7 @@ bwd_owner_kernel(const float *__restrict__ v, const float *__restrict__ g, float
             k[i][j] = K[c * (B * B) + i * B + j];
             acc[i][j] = 0.0;
         }
+    prior_kernel_done();
     const int64_t alpha = c / s, base = alpha * B * s + (c - alpha * s);
     constexpr int U = B >= 7 ? 2 : kRowBatch;         // radices 7 and 8 already fill the register file
     const int64_t r0 = (int64_t)blockIdx.y * kBwdSliceRows, r1 = min(rows, r0 + kBwdSliceRows);
@@ -174,6 +204,7 @@ stage16_kernel(const float *__restrict__ in, float *__restrict__ out, int64_t ro
     for (int q = 0; q < 16; ++q)
 #pragma unroll
         for (int t = 0; t < 4; ++t) k[q][t] = K[c * 256 + (transpose ? (t0 + t) * 16 + q : q * 16 + t0 + t)];
+    prior_kernel_done();
     const int64_t alpha = c / s, base = alpha * 16 * s + (c - alpha * s);
     const int64_t r0 = (int64_t)blockIdx.y * kFwdSliceRows, r1 = min(rows, r0 + kFwdSliceRows);
 #pragma unroll 2
@@ -209,6 +240,7 @@ outer16_kernel(const float *__restrict__ v, const float *__restrict__ g, int64_t
     for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.0;
+    prior_kernel_done();
     const int64_t alpha = c / s, base = alpha * 16 * s + (c - alpha * s);
     const int64_t r0 = (int64_t)blockIdx.y * kTileRows16, r1 = min(rows, r0 + kTileRows16);
     for (int64_t r = r0; r < r1; r += 2) {
@@ -241,6 +273,7 @@ outer16_kernel(const float *__restrict__ v, const float *__restrict__ g, int64_t
 __global__ void __launch_bounds__(kThreads)
 reduce_slices_kernel(const double *__restrict__ part, int64_t n_slices, int64_t nblk, int bb, float *__restrict__ grad,
                      int accumulate) {
+    prior_kernel_done();
     __shared__ double warp_sum[kThreads / 32][32];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int64_t total = nblk * bb;
@@ -274,6 +307,7 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads)
 load_rows_kernel(const T *__restrict__ x, const T *__restrict__ gy, int64_t rows, int64_t d, const int32_t *__restrict__ perm,
                  const int8_t *__restrict__ signs, float *__restrict__ v0, float *__restrict__ g) {
+    prior_kernel_done();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     T *row = reinterpret_cast<T *>(smem_raw);
     for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
@@ -294,6 +328,7 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads)
 load_kernel(const T *__restrict__ x, const T *__restrict__ gy, int64_t rows, int64_t d, const int32_t *__restrict__ perm,
             const int8_t *__restrict__ signs, float *__restrict__ v0, float *__restrict__ g) {
+    prior_kernel_done();
     const int64_t total = rows * d;
     for (int64_t e = (int64_t)blockIdx.x * kThreads + threadIdx.x; e < total; e += (int64_t)gridDim.x * kThreads) {
         const int64_t r = e / d, i = e - r * d;
@@ -311,6 +346,7 @@ load_kernel(const T *__restrict__ x, const T *__restrict__ gy, int64_t rows, int
 __global__ void __launch_bounds__(kThreads)
 stage_kernel(const float *__restrict__ in, float *__restrict__ out, int64_t rows, int64_t d, int b, int64_t s,
              const float *__restrict__ K, int64_t kc_step, int64_t kk_step, int transpose) {
+    prior_kernel_done();
     const int64_t total = rows * d;
     for (int64_t e = (int64_t)blockIdx.x * kThreads + threadIdx.x; e < total; e += (int64_t)gridDim.x * kThreads) {
         const int64_t r = e / d, pos = e - r * d;
@@ -334,6 +370,7 @@ stage_kernel(const float *__restrict__ in, float *__restrict__ out, int64_t rows
 __global__ void __launch_bounds__(kThreads)
 outer_kernel(const float *__restrict__ v, const float *__restrict__ g, int64_t rows, int64_t d, int b, int64_t s,
              float *__restrict__ grad, int accumulate, int by_block) {
+    prior_kernel_done();
     __shared__ double part[kThreads / 32][32];
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int64_t total = d * b;                       // (d / b) blocks of b*b entries
@@ -362,6 +399,33 @@ outer_kernel(const float *__restrict__ v, const float *__restrict__ g, int64_t r
     }
 }
 
+// Scratch comes from a memory pool of the library's own (one per device, created on first use)
+// whose release threshold is unlimited: the default pool hands its memory back at every
+// synchronisation, and mapping 256 MB anew costs more than the kernels of a call.  Returns null
+// if the pool cannot be created; the caller then allocates from the device's default pool.
+cudaMemPool_t scratch_pool(int device) {
+    static std::mutex mu;
+    static std::map<int, cudaMemPool_t> pools;
+    std::lock_guard<std::mutex> lock(mu);
+    auto it = pools.find(device);
+    if (it != pools.end()) return it->second;
+    cudaMemPoolProps props = {};
+    props.allocType = cudaMemAllocationTypePinned;
+    props.handleTypes = cudaMemHandleTypeNone;
+    props.location.type = cudaMemLocationTypeDevice;
+    props.location.id = device;
+    cudaMemPool_t pool = nullptr;
+    if (cudaMemPoolCreate(&pool, &props) != cudaSuccess) {
+        cudaGetLastError();
+        pool = nullptr;
+    } else {
+        uint64_t keep = ~0ull;
+        cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+    }
+    pools[device] = pool;
+    return pool;
+}
+
 unsigned grid_for(int64_t work) {
     return (unsigned)std::max<int64_t>(1, std::min<int64_t>((work + kThreads - 1) / kThreads, 148 * 16));
 }
@@ -379,13 +443,13 @@ dim3 owner_grid(int64_t d, int b, int64_t rows, int slice_rows) {
 void launch_fwd_owner(int b, const float *in, float *out, int64_t rows, int64_t d, int64_t s, const float *K, cudaStream_t st) {
     const dim3 grid = owner_grid(d, b, rows, kFwdSliceRows);
     switch (b) {
-        case 2: fwd_owner_kernel<2><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K); break;
-        case 3: fwd_owner_kernel<3><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K); break;
-        case 4: fwd_owner_kernel<4><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K); break;
-        case 5: fwd_owner_kernel<5><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K); break;
-        case 6: fwd_owner_kernel<6><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K); break;
-        case 7: fwd_owner_kernel<7><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K); break;
-        default: fwd_owner_kernel<8><<<grid, kOwnThreads, 0, st>>>(in, out, rows, d, s, K); break;
+        case 2: launch_dep(fwd_owner_kernel<2>, dim3(grid), dim3(kOwnThreads), 0, st, in, out, rows, d, s, K); break;
+        case 3: launch_dep(fwd_owner_kernel<3>, dim3(grid), dim3(kOwnThreads), 0, st, in, out, rows, d, s, K); break;
+        case 4: launch_dep(fwd_owner_kernel<4>, dim3(grid), dim3(kOwnThreads), 0, st, in, out, rows, d, s, K); break;
+        case 5: launch_dep(fwd_owner_kernel<5>, dim3(grid), dim3(kOwnThreads), 0, st, in, out, rows, d, s, K); break;
+        case 6: launch_dep(fwd_owner_kernel<6>, dim3(grid), dim3(kOwnThreads), 0, st, in, out, rows, d, s, K); break;
+        case 7: launch_dep(fwd_owner_kernel<7>, dim3(grid), dim3(kOwnThreads), 0, st, in, out, rows, d, s, K); break;
+        default: launch_dep(fwd_owner_kernel<8>, dim3(grid), dim3(kOwnThreads), 0, st, in, out, rows, d, s, K); break;
     }
 }
 
@@ -393,13 +457,13 @@ void launch_bwd_owner(int b, const float *v, const float *g, float *g_out, int64
                       double *part, cudaStream_t st) {
     const dim3 grid = owner_grid(d, b, rows, kBwdSliceRows);
     switch (b) {
-        case 2: bwd_owner_kernel<2><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part); break;
-        case 3: bwd_owner_kernel<3><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part); break;
-        case 4: bwd_owner_kernel<4><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part); break;
-        case 5: bwd_owner_kernel<5><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part); break;
-        case 6: bwd_owner_kernel<6><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part); break;
-        case 7: bwd_owner_kernel<7><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part); break;
-        default: bwd_owner_kernel<8><<<grid, kOwnThreads, 0, st>>>(v, g, g_out, rows, d, s, K, part); break;
+        case 2: launch_dep(bwd_owner_kernel<2>, dim3(grid), dim3(kOwnThreads), 0, st, v, g, g_out, rows, d, s, K, part); break;
+        case 3: launch_dep(bwd_owner_kernel<3>, dim3(grid), dim3(kOwnThreads), 0, st, v, g, g_out, rows, d, s, K, part); break;
+        case 4: launch_dep(bwd_owner_kernel<4>, dim3(grid), dim3(kOwnThreads), 0, st, v, g, g_out, rows, d, s, K, part); break;
+        case 5: launch_dep(bwd_owner_kernel<5>, dim3(grid), dim3(kOwnThreads), 0, st, v, g, g_out, rows, d, s, K, part); break;
+        case 6: launch_dep(bwd_owner_kernel<6>, dim3(grid), dim3(kOwnThreads), 0, st, v, g, g_out, rows, d, s, K, part); break;
+        case 7: launch_dep(bwd_owner_kernel<7>, dim3(grid), dim3(kOwnThreads), 0, st, v, g, g_out, rows, d, s, K, part); break;
+        default: launch_dep(bwd_owner_kernel<8>, dim3(grid), dim3(kOwnThreads), 0, st, v, g, g_out, rows, d, s, K, part); break;
     }
 }
 
@@ -409,10 +473,10 @@ void launch_load(const T *x, const T *gy, int64_t rows, int64_t d, const harp_pl
     static const bool big_ok =
         cudaFuncSetAttribute(load_rows_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) == cudaSuccess;
     if (plan->d_perm && (smem <= 48 * 1024 || (big_ok && smem <= 200 * 1024)))
-        load_rows_kernel<T><<<(unsigned)std::min<int64_t>(rows, 148 * 8), kThreads, smem, st>>>(x, gy, rows, d, plan->d_perm,
-                                                                                                 plan->d_signs, v0, g);
+        launch_dep(load_rows_kernel<T>, dim3((unsigned)std::min<int64_t>(rows, 148 * 8)), dim3(kThreads), smem, st, x, gy, rows, d,
+                   plan->d_perm, plan->d_signs, v0, g);
     else
-        load_kernel<T><<<grid_for(rows * d), kThreads, 0, st>>>(x, gy, rows, d, plan->d_perm, plan->d_signs, v0, g);
+        launch_dep(load_kernel<T>, dim3(grid_for(rows * d)), dim3(kThreads), 0, st, x, gy, rows, d, plan->d_perm, plan->d_signs, v0, g);
 }
 
 }  // namespace
@@ -447,7 +511,11 @@ extern "C" harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x
     }
     const int64_t state_bytes = (int64_t)(m + 2) * chunk * d * (int64_t)sizeof(float);
     float *scratch = nullptr;
-    if (cudaMallocAsync(reinterpret_cast<void **>(&scratch), (size_t)(state_bytes + 256 + part_bytes), st) != cudaSuccess) {
+    const size_t scratch_bytes = (size_t)(state_bytes + 256 + part_bytes);
+    cudaMemPool_t pool = scratch_pool(plan->device);
+    const cudaError_t alloc_err = pool ? cudaMallocFromPoolAsync(reinterpret_cast<void **>(&scratch), scratch_bytes, pool, st)
+                                       : cudaMallocAsync(reinterpret_cast<void **>(&scratch), scratch_bytes, st);
+    if (alloc_err != cudaSuccess) {
         cudaGetLastError();
         return HARP_ERR_ALLOC;
     }
@@ -469,12 +537,17 @@ extern "C" harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x
         for (int t = 0; t + 1 < m; ++t, ++launches) {
             const int b = plan->st.b[t];
             const float *K = plan->d_blocks + plan->st.off[t];
-            const bool em = plan->st.s[t] >= 8;             // see stage_kernel
-            if (owner_radix(b)) launch_fwd_owner(b, scratch + t * plane, scratch + (t + 1) * plane, rows, d, plan->st.s[t], K, st);
-            else if (b == 16) stage16_kernel<<<owner_grid16(d, rows, kFwdSliceRows), 128, 0, st>>>(scratch + t * plane, scratch + (t + 1) * plane, rows, d, plan->st.s[t], K, 0);
-            else stage_kernel<<<grid, kThreads, 0, st>>>(scratch + t * plane, scratch + (t + 1) * plane, rows, d, b, plan->st.s[t],
-                                                         em ? plan->d_blocks_em + plan->st.off[t] : K, em ? 1 : (int64_t)b * b,
-                                                         em ? d / b : 1, 0);
+            const int64_t s = plan->st.s[t];
+            const bool em = s >= 8;                          // see stage_kernel
+            const float *v_in = scratch + t * plane;
+            float *v_out = scratch + (t + 1) * plane;
+            if (owner_radix(b))
+                launch_fwd_owner(b, v_in, v_out, rows, d, s, K, st);
+            else if (b == 16)
+                launch_dep(stage16_kernel, owner_grid16(d, rows, kFwdSliceRows), dim3(128), 0, st, v_in, v_out, rows, d, s, K, 0);
+            else
+                launch_dep(stage_kernel, dim3(grid), dim3(kThreads), 0, st, v_in, v_out, rows, d, b, s,
+                           em ? plan->d_blocks_em + plan->st.off[t] : K, em ? 1 : (int64_t)b * b, em ? d / b : 1, 0);
         }
         // backward: entry sums, and the gradient state one stage back
         float *g_cur = ga, *g_nxt = gb;
@@ -483,24 +556,28 @@ extern "C" harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x
             const int b = plan->st.b[t];
             const int64_t s = plan->st.s[t];
             const float *K = plan->d_blocks + plan->st.off[t];
+            const float *v_t = scratch + t * plane;
+            float *grad_t = grad + plan->st.off[t];
+            const dim3 reduce_grid((unsigned)std::min<int64_t>((d * b + 31) / 32, 148 * 16));
             if (owner_radix(b)) {
-                launch_bwd_owner(b, scratch + t * plane, g_cur, t > 0 ? g_nxt : nullptr, rows, d, s, K, part, st);
-                reduce_slices_kernel<<<(unsigned)std::min<int64_t>((d * b + 31) / 32, 148 * 16), kThreads, 0, st>>>(part, (rows + kBwdSliceRows - 1) / kBwdSliceRows, d / b, b * b,
-                                                                           grad + plan->st.off[t], acc);
+                launch_bwd_owner(b, v_t, g_cur, t > 0 ? g_nxt : nullptr, rows, d, s, K, part, st);
+                launch_dep(reduce_slices_kernel, reduce_grid, dim3(kThreads), 0, st, part, (rows + kBwdSliceRows - 1) / kBwdSliceRows,
+                           d / b, b * b, grad_t, acc);
                 launches += 2;
             } else if (b == 16) {
-                outer16_kernel<<<owner_grid16(d, rows, kTileRows16), 512, 0, st>>>(scratch + t * plane, g_cur, rows, d, s, part);
-                reduce_slices_kernel<<<(unsigned)std::min<int64_t>((d * b + 31) / 32, 148 * 16), kThreads, 0, st>>>(
-                    part, (rows + kTileRows16 - 1) / kTileRows16, d / b, b * b, grad + plan->st.off[t], acc);
-                if (t > 0) stage16_kernel<<<owner_grid16(d, rows, kFwdSliceRows), 128, 0, st>>>(g_cur, g_nxt, rows, d, s, K, 1);
+                launch_dep(outer16_kernel, owner_grid16(d, rows, kTileRows16), dim3(512), 0, st, v_t, g_cur, rows, d, s, part);
+                launch_dep(reduce_slices_kernel, reduce_grid, dim3(kThreads), 0, st, part, (rows + kTileRows16 - 1) / kTileRows16,
+                           d / b, b * b, grad_t, acc);
+                if (t > 0)
+                    launch_dep(stage16_kernel, owner_grid16(d, rows, kFwdSliceRows), dim3(128), 0, st, g_cur, g_nxt, rows, d, s, K, 1);
                 launches += t > 0 ? 3 : 2;
             } else {
                 const bool em = s >= 8;
-                outer_kernel<<<(unsigned)std::min<int64_t>((d * b + 31) / 32, 148 * 64), kThreads, 0, st>>>(
-                    scratch + t * plane, g_cur, rows, d, b, s, grad + plan->st.off[t], acc, em ? 0 : 1);
+                launch_dep(outer_kernel, dim3((unsigned)std::min<int64_t>((d * b + 31) / 32, 148 * 64)), dim3(kThreads), 0, st, v_t,
+                           g_cur, rows, d, b, s, grad_t, acc, em ? 0 : 1);
                 if (t > 0)
-                    stage_kernel<<<grid, kThreads, 0, st>>>(g_cur, g_nxt, rows, d, b, s, em ? plan->d_blocks_em + plan->st.off[t] : K,
-                                                            em ? 1 : (int64_t)b * b, em ? d / b : 1, 1);
+                    launch_dep(stage_kernel, dim3(grid), dim3(kThreads), 0, st, g_cur, g_nxt, rows, d, b, s,
+                               em ? plan->d_blocks_em + plan->st.off[t] : K, em ? 1 : (int64_t)b * b, em ? d / b : 1, 1);
                 launches += t > 0 ? 2 : 1;
             }
             if (t > 0) std::swap(g_cur, g_nxt);
