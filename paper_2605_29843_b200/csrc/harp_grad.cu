@@ -58,7 +58,7 @@ template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16
 
 constexpr int kOwnThreads = 128;   // block-owner kernels: blocks per CTA
 constexpr int kFwdSliceRows = 8;   //                      rows per CTA, forward
-constexpr int kBwdSliceRows = 16;  //                      rows per CTA (one set of partial sums), backward
+constexpr int kBwdSliceRows = 32;  //                      rows per CTA (one set of partial sums), backward
 constexpr int kRowBatch = 4;       //                      rows whose loads are issued together
 
 template <int B> __device__ __forceinline__ void load_block(const float *p, int64_t s, float (&v)[B]) {
@@ -500,7 +500,7 @@ extern "C" harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x
         return HARP_OK;
     }
     // chunk of rows whose m forward states, two gradient states and the per-slice sums of the
-    // block-owner stages (at most one state: 8 bytes x d b / 16 per row for b <= 8, d b / 32 for b = 16) fit ~256 MB
+    // block-owner stages (at most one state: 8 bytes x d b / 32 per row, b <= 16) fit ~256 MB
     const int64_t per_row = (int64_t)(m + 3) * d * (int64_t)sizeof(float);
     const int64_t chunk = std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(n_rows, 1 << 18), (256ll << 20) / per_row));
     int64_t part_bytes = 0;                          // per-slice sums of the stage that needs most
