@@ -109,6 +109,30 @@ def test_euler_identity_at_full_dimension():
     assert off == grad.numel()
 
 
+@pytest.mark.parametrize("cfg", [3, 4, 5])
+def test_euler_identity_on_the_wide_plans(cfg):
+    """The wide configurations' plans at full dimension (radices 2 and 43; 16, 16, 8, 7; 8, 8, 8, 8, 2),
+    bf16 rows: <K_t, dL/dK_t> = L = sum(y * G) for every stage, with y from the fp64 oracle."""
+    w = wl.config(cfg)
+    spec = list(w.plans.values())[0]
+    plan = harp.plan_from_spec(spec)
+    oplan = orc.OraclePlan.from_spec(spec)
+    rng = np.random.default_rng(80 + cfg)
+    n = 96
+    xh = host_rows(rng.standard_normal((n, spec.d)), "bf16")
+    gh = host_rows(rng.standard_normal((n, spec.d)), "bf16")
+    grad, _, _ = _gpu_grad(plan, xh, gh, "bf16")
+    L = float(np.sum(orc.forward(oplan, promote(xh, "bf16")) * promote(gh, "bf16")))
+    scale = float(np.sqrt(n * spec.d))                      # size of L for independent unit-variance terms
+    off = 0
+    for t, b in enumerate(spec.radices):
+        k = np.asarray(spec.blocks[t], dtype=np.float32).astype(np.float64).ravel()
+        got = float(np.dot(k, grad[off:off + k.size]))
+        off += k.size
+        assert abs(got - L) <= 2e-4 * max(abs(L), scale), (t, b, got, L)
+    assert off == grad.size
+
+
 def test_parameter_gradient_of_a_plan_built_from_theta():
     """One parameter step's worth of Algorithm 3 without the quantizer: plan from theta, L = sum(y * G)
     with y from harp_apply, dL/dK on the GPU, dL/dtheta on the host; compared with central
