@@ -58,32 +58,36 @@ __device__ void cta_accumulate(double v, double *dst, bool is_max) {
 }
 
 // acc[1] = max |a|, acc[2] = sum a^2, acc[3] = sum of a^2 over the diagonal blocks (block > 0)
-template <typename T, int V>
+// BLOCKS: also sum the squares inside the diagonal blocks (off-block energy); without it the loop
+// spends one conversion and one fp64 multiply-add per element (the maximum is taken in fp32,
+// which is exact for fp32 and bf16 inputs) -- fp64 issue is what bounds this kernel.
+template <typename T, int V, bool BLOCKS>
 __global__ void __launch_bounds__(kThreads)
 stats_kernel(const T *__restrict__ A, int64_t m, int64_t n, int64_t block, double *acc) {
     const int64_t c0 = ((int64_t)blockIdx.x * kThreads + threadIdx.x) * V;
-    double mx = 0.0, ss = 0.0, sd = 0.0;
+    float mxf = 0.f;
+    double ss = 0.0, sd = 0.0;
     if (c0 < n) {
         int64_t cb[V];
 #pragma unroll
-        for (int v = 0; v < V; ++v) cb[v] = block > 0 ? (c0 + v) / block : -1;
+        for (int v = 0; v < V; ++v) cb[v] = BLOCKS ? (c0 + v) / block : -1;
 #pragma unroll 4
         for (int64_t r = blockIdx.y; r < m; r += gridDim.y) {
-            const int64_t rb = block > 0 ? r / block : -2;
+            const int64_t rb = BLOCKS ? r / block : -2;
             float a[V];
             load_vec<T, V>(A + r * n + c0, a);
 #pragma unroll
             for (int v = 0; v < V; ++v) {
                 const double x = (double)a[v];
-                mx = fmax(mx, fabs(x));
+                mxf = fmaxf(mxf, fabsf(a[v]));
                 ss += x * x;
-                if (cb[v] == rb) sd += x * x;
+                if (BLOCKS && cb[v] == rb) sd += x * x;
             }
         }
     }
-    cta_accumulate(mx, acc + 1, true);
+    cta_accumulate((double)mxf, acc + 1, true);
     cta_accumulate(ss, acc + 2, false);
-    if (block > 0) cta_accumulate(sd, acc + 3, false);
+    if (BLOCKS) cta_accumulate(sd, acc + 3, false);
 }
 
 // acc[1] = sum_ij (Wt_ij - Wq_ij)^2 |H_jj|, acc[2] = sum_j |H_jj| (added by the CTAs of row class 0 only)
@@ -148,17 +152,23 @@ harp_status_t check_common(const void *A, int64_t m, int64_t n, harp_dtype_t dty
     return HARP_OK;
 }
 
+template <typename T, int V>
+void launch_stats(bool vec, const T *A, int64_t m, int64_t n, int64_t block, double *out, cudaStream_t stream) {
+    if (vec && block > 0) stats_kernel<T, V, true><<<grid_for(m, n, V), kThreads, 0, stream>>>(A, m, n, block, out);
+    else if (vec) stats_kernel<T, V, false><<<grid_for(m, n, V), kThreads, 0, stream>>>(A, m, n, block, out);
+    else if (block > 0) stats_kernel<T, 1, true><<<grid_for(m, n, 1), kThreads, 0, stream>>>(A, m, n, block, out);
+    else stats_kernel<T, 1, false><<<grid_for(m, n, 1), kThreads, 0, stream>>>(A, m, n, block, out);
+}
+
 harp_status_t run_stats(const void *A, int64_t m, int64_t n, int64_t block, harp_dtype_t dtype, double *out,
                         int final_kind, cudaStream_t stream) {
     if (cudaMemsetAsync(out, 0, 4 * sizeof(double), stream) != cudaSuccess) return HARP_ERR_CUDA;
     const int V = dtype == HARP_F32 ? 4 : 8;
     const bool vec = aligned16(A) && n % V == 0;
     if (dtype == HARP_F32) {
-        if (vec) stats_kernel<float, 4><<<grid_for(m, n, 4), kThreads, 0, stream>>>((const float *)A, m, n, block, out);
-        else stats_kernel<float, 1><<<grid_for(m, n, 1), kThreads, 0, stream>>>((const float *)A, m, n, block, out);
+        launch_stats<float, 4>(vec, (const float *)A, m, n, block, out, stream);
     } else {
-        if (vec) stats_kernel<__nv_bfloat16, 8><<<grid_for(m, n, 8), kThreads, 0, stream>>>((const __nv_bfloat16 *)A, m, n, block, out);
-        else stats_kernel<__nv_bfloat16, 1><<<grid_for(m, n, 1), kThreads, 0, stream>>>((const __nv_bfloat16 *)A, m, n, block, out);
+        launch_stats<__nv_bfloat16, 8>(vec, (const __nv_bfloat16 *)A, m, n, block, out, stream);
     }
     finalize_kernel<<<1, 1, 0, stream>>>(out, final_kind, (double)m, (double)n);
     g_harp_launches.fetch_add(2, std::memory_order_relaxed);
