@@ -310,14 +310,51 @@ load_rows_kernel(const T *__restrict__ x, const T *__restrict__ gy, int64_t rows
     prior_kernel_done();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     T *row = reinterpret_cast<T *>(smem_raw);
+    constexpr int V = 16 / (int)sizeof(T);                 // elements per 16-byte access
+    // 16-byte accesses when every row starts on a 16-byte boundary; V divides 64, so the V elements
+    // of one access stay next to each other in the staged row
+    const bool vec = d % V == 0 && ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(gy)) & 15) == 0;
     for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
-        for (int64_t i = threadIdx.x; i < d; i += kThreads) row[staged_pos(i)] = x[r * d + i];
+        if (vec) {
+            for (int64_t i = (int64_t)threadIdx.x * V; i < d; i += (int64_t)kThreads * V) {
+                const uint4 raw = *reinterpret_cast<const uint4 *>(x + r * d + i);
+                const uint32_t *w = reinterpret_cast<const uint32_t *>(&raw);
+                uint32_t *dst = reinterpret_cast<uint32_t *>(row + staged_pos(i));   // 4-byte aligned: staged_pos(i) is even
+#pragma unroll
+                for (int k = 0; k < 4; ++k) dst[k] = w[k];
+                const uint4 rg = *reinterpret_cast<const uint4 *>(gy + r * d + i);
+                const T *tg = reinterpret_cast<const T *>(&rg);
+                float *gd = g + r * d + i;
+#pragma unroll
+                for (int k = 0; k < V; k += 4)
+                    *reinterpret_cast<float4 *>(gd + k) =
+                        make_float4(to_f32<T>(tg[k]), to_f32<T>(tg[k + 1]), to_f32<T>(tg[k + 2]), to_f32<T>(tg[k + 3]));
+            }
+        } else {
+            for (int64_t i = threadIdx.x; i < d; i += kThreads) {
+                row[staged_pos(i)] = x[r * d + i];
+                g[r * d + i] = to_f32<T>(gy[r * d + i]);
+            }
+        }
         __syncthreads();
-        for (int64_t i = threadIdx.x; i < d; i += kThreads) {
-            const int64_t src = perm[i];
-            const float sg = (signs && signs[src] < 0) ? -1.f : 1.f;
-            v0[r * d + i] = sg * to_f32<T>(row[staged_pos(src)]);
-            g[r * d + i] = to_f32<T>(gy[r * d + i]);
+        if (d % 4 == 0) {
+            for (int64_t i = (int64_t)threadIdx.x * 4; i < d; i += (int64_t)kThreads * 4) {
+                const int4 src = *reinterpret_cast<const int4 *>(perm + i);
+                const int sidx[4] = {src.x, src.y, src.z, src.w};
+                float o[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const float sg = (signs && signs[sidx[k]] < 0) ? -1.f : 1.f;
+                    o[k] = sg * to_f32<T>(row[staged_pos(sidx[k])]);
+                }
+                *reinterpret_cast<float4 *>(v0 + r * d + i) = make_float4(o[0], o[1], o[2], o[3]);
+            }
+        } else {
+            for (int64_t i = threadIdx.x; i < d; i += kThreads) {
+                const int64_t src = perm[i];
+                const float sg = (signs && signs[src] < 0) ? -1.f : 1.f;
+                v0[r * d + i] = sg * to_f32<T>(row[staged_pos(src)]);
+            }
         }
         __syncthreads();
     }
