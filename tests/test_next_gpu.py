@@ -109,3 +109,41 @@ def test_passes(dtype):
     with pytest.raises(harp.HarpError):
         harp.harp_apply_passes([plans[0], harp.plan_from_spec(wl.tiny_plan(1, (4, 4), kind="qr"))],
                                to_device(xh, dtype).data_ptr(), 33, code)
+
+
+@pytest.mark.parametrize("n_rows", [1, 16, 64])
+def test_small_batches_chained_and_in_a_cuda_graph(n_rows):
+    """Wide rows, few rows (the decode case): consecutive applies on a side stream overlap each
+    kernel's preamble with the kernel before it.  A forward/transpose chain must give the same bits
+    whether launched call by call or replayed from a CUDA graph, and match the oracle."""
+    w = wl.config(4)
+    spec = w.plans["q"]
+    plan = harp.plan_from_spec(spec)
+    oplan = orc.OraclePlan.from_spec(spec)
+    rng = np.random.default_rng(90 + n_rows)
+    xh = host_rows(rng.standard_normal((n_rows, spec.d)), "bf16")
+    side = torch.cuda.Stream()
+
+    def chain(x, st):
+        for k in range(5):                                  # F T F T F: one forward in total
+            harp.harp_apply(plan, x.data_ptr(), n_rows, harp.HARP_BF16, bool(k & 1), st)
+
+    eager = to_device(xh, "bf16")
+    with torch.cuda.stream(side):
+        chain(eager, side.cuda_stream)
+    side.synchronize()
+    replayed = to_device(xh, "bf16")
+    graph = torch.cuda.CUDAGraph()
+    scratch = to_device(xh, "bf16")
+    with torch.cuda.stream(side):
+        chain(scratch, side.cuda_stream)                    # warm-up before capture
+        side.synchronize()
+        scratch.copy_(replayed)
+        with torch.cuda.graph(graph, stream=side):
+            chain(scratch, side.cuda_stream)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(eager.view(torch.int16), scratch.view(torch.int16))
+    # five roundings to bf16 along the chain: a few times the single-apply tolerance
+    want = orc.forward(oplan, promote(xh, "bf16"))
+    assert orc.rel_err_rows(to_host_f64(eager), want) <= 3 * TOL["bf16"]
