@@ -68,21 +68,26 @@ stats_kernel(const T *__restrict__ A, int64_t m, int64_t n, int64_t block, doubl
     float mxf = 0.f;
     double ss = 0.0, sd = 0.0;
     if (c0 < n) {
-        int64_t cb[V];
+        int64_t lo[V];                                    // first row of the diagonal block of column c0 + v
 #pragma unroll
-        for (int v = 0; v < V; ++v) cb[v] = BLOCKS ? (c0 + v) / block : -1;
+        for (int v = 0; v < V; ++v) lo[v] = BLOCKS ? (c0 + v) / block * block : 0;
+        // c0 is a multiple of V: when V divides the block size the thread's V columns share a block
+        // and one comparison per row decides whether the row's partial sum is inside it
+        const bool one_block = BLOCKS && block % V == 0;
 #pragma unroll 4
         for (int64_t r = blockIdx.y; r < m; r += gridDim.y) {
-            const int64_t rb = BLOCKS ? r / block : -2;
             float a[V];
             load_vec<T, V>(A + r * n + c0, a);
+            double row_ss = 0.0, row_sd = 0.0;
 #pragma unroll
             for (int v = 0; v < V; ++v) {
                 const double x = (double)a[v];
                 mxf = fmaxf(mxf, fabsf(a[v]));
-                ss += x * x;
-                if (BLOCKS && cb[v] == rb) sd += x * x;
+                row_ss += x * x;
+                if (BLOCKS && !one_block && r >= lo[v] && r < lo[v] + block) row_sd += x * x;
             }
+            ss += row_ss;
+            if (BLOCKS) sd += one_block ? ((r >= lo[0] && r < lo[0] + block) ? row_ss : 0.0) : row_sd;
         }
     }
     cta_accumulate((double)mxf, acc + 1, true);
