@@ -366,13 +366,14 @@ __global__ void __launch_bounds__(kThreads)
 load_kernel(const T *__restrict__ x, const T *__restrict__ gy, int64_t rows, int64_t d, const int32_t *__restrict__ perm,
             const int8_t *__restrict__ signs, float *__restrict__ v0, float *__restrict__ g) {
     prior_kernel_done();
-    const int64_t total = rows * d;
-    for (int64_t e = (int64_t)blockIdx.x * kThreads + threadIdx.x; e < total; e += (int64_t)gridDim.x * kThreads) {
-        const int64_t r = e / d, i = e - r * d;
-        const int64_t src = perm ? perm[i] : i;
-        const float sg = (signs && signs[src] < 0) ? -1.f : 1.f;
-        v0[e] = sg * to_f32<T>(x[r * d + src]);
-        g[e] = to_f32<T>(gy[e]);
+    // a thread keeps its coordinate and walks over rows (blockIdx.y, then in steps of gridDim.y)
+    const int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (i >= d) return;
+    const int64_t src = perm ? perm[i] : i;
+    const float sg = (signs && signs[src] < 0) ? -1.f : 1.f;
+    for (int64_t r = blockIdx.y; r < rows; r += gridDim.y) {
+        v0[r * d + i] = sg * to_f32<T>(x[r * d + src]);
+        g[r * d + i] = to_f32<T>(gy[r * d + i]);
     }
 }
 
@@ -384,18 +385,19 @@ __global__ void __launch_bounds__(kThreads)
 stage_kernel(const float *__restrict__ in, float *__restrict__ out, int64_t rows, int64_t d, int b, int64_t s,
              const float *__restrict__ K, int64_t kc_step, int64_t kk_step, int transpose) {
     prior_kernel_done();
-    const int64_t total = rows * d;
-    for (int64_t e = (int64_t)blockIdx.x * kThreads + threadIdx.x; e < total; e += (int64_t)gridDim.x * kThreads) {
-        const int64_t r = e / d, pos = e - r * d;
-        const int64_t alpha = pos / (b * s), rem = pos - alpha * b * s;
-        const int64_t j = rem / s, beta = rem - j * s;
-        const int64_t base = alpha * b * s + beta;
-        const float *Kc = K + (alpha * s + beta) * kc_step;
+    // a thread keeps its position (the index arithmetic is done once) and walks over rows
+    const int64_t pos = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+    if (pos >= d) return;
+    const int64_t alpha = pos / (b * s), rem = pos - alpha * b * s;
+    const int64_t j = rem / s, beta = rem - j * s;
+    const int64_t base = alpha * b * s + beta;
+    const float *Kc = K + (alpha * s + beta) * kc_step + (transpose ? j * b : j) * kk_step;
+    const int64_t k_step = (transpose ? 1 : (int64_t)b) * kk_step;     // from K[..][i][j] to K[..][i+1][j] (or [j][i+1])
+    for (int64_t r = blockIdx.y; r < rows; r += gridDim.y) {
         const float *row = in + r * d + base;
         float acc = 0.f;
-        for (int i = 0; i < b; ++i)
-            acc = fmaf(row[(int64_t)i * s], Kc[(transpose ? j * b + i : (int64_t)i * b + j) * kk_step], acc);
-        out[e] = acc;
+        for (int i = 0; i < b; ++i) acc = fmaf(row[(int64_t)i * s], Kc[(int64_t)i * k_step], acc);
+        out[r * d + pos] = acc;
     }
 }
 
@@ -463,8 +465,11 @@ cudaMemPool_t scratch_pool(int device) {
     return pool;
 }
 
-unsigned grid_for(int64_t work) {
-    return (unsigned)std::max<int64_t>(1, std::min<int64_t>((work + kThreads - 1) / kThreads, 148 * 16));
+// grid of the kernels in which a thread keeps its coordinate and walks over rows
+dim3 column_grid(int64_t d, int64_t rows) {
+    const int64_t gx = (d + kThreads - 1) / kThreads;
+    const int64_t gy = std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(rows, 65535), (148 * 16 + gx - 1) / gx));
+    return dim3((unsigned)gx, (unsigned)gy);
 }
 
 bool owner_radix(int b) { return b >= 2 && b <= 8; }
@@ -513,7 +518,7 @@ void launch_load(const T *x, const T *gy, int64_t rows, int64_t d, const harp_pl
         launch_dep(load_rows_kernel<T>, dim3((unsigned)std::min<int64_t>(rows, 148 * 8)), dim3(kThreads), smem, st, x, gy, rows, d,
                    plan->d_perm, plan->d_signs, v0, g);
     else
-        launch_dep(load_kernel<T>, dim3(grid_for(rows * d)), dim3(kThreads), 0, st, x, gy, rows, d, plan->d_perm, plan->d_signs, v0, g);
+        launch_dep(load_kernel<T>, column_grid(d, rows), dim3(kThreads), 0, st, x, gy, rows, d, plan->d_perm, plan->d_signs, v0, g);
 }
 
 }  // namespace
@@ -563,7 +568,6 @@ extern "C" harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x
     harp_status_t rc = HARP_OK;
     for (int64_t r0 = 0; r0 < n_rows && rc == HARP_OK; r0 += chunk) {
         const int64_t rows = std::min(chunk, n_rows - r0);
-        const unsigned grid = grid_for(rows * d);
         if (dtype == HARP_F32)
             launch_load<float>((const float *)x + r0 * d, (const float *)gy + r0 * d, rows, d, plan, scratch, ga, st);
         else
@@ -583,7 +587,7 @@ extern "C" harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x
             else if (b == 16)
                 launch_dep(stage16_kernel, owner_grid16(d, rows, kFwdSliceRows), dim3(128), 0, st, v_in, v_out, rows, d, s, K, 0);
             else
-                launch_dep(stage_kernel, dim3(grid), dim3(kThreads), 0, st, v_in, v_out, rows, d, b, s,
+                launch_dep(stage_kernel, column_grid(d, rows), dim3(kThreads), 0, st, v_in, v_out, rows, d, b, s,
                            em ? plan->d_blocks_em + plan->st.off[t] : K, em ? 1 : (int64_t)b * b, em ? d / b : 1, 0);
         }
         // backward: entry sums, and the gradient state one stage back
@@ -613,7 +617,7 @@ extern "C" harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x
                 launch_dep(outer_kernel, dim3((unsigned)std::min<int64_t>((d * b + 31) / 32, 148 * 64)), dim3(kThreads), 0, st, v_t,
                            g_cur, rows, d, b, s, grad_t, acc, em ? 0 : 1);
                 if (t > 0)
-                    launch_dep(stage_kernel, dim3(grid), dim3(kThreads), 0, st, g_cur, g_nxt, rows, d, b, s,
+                    launch_dep(stage_kernel, column_grid(d, rows), dim3(kThreads), 0, st, g_cur, g_nxt, rows, d, b, s,
                                em ? plan->d_blocks_em + plan->st.off[t] : K, em ? 1 : (int64_t)b * b, em ? d / b : 1, 1);
                 launches += t > 0 ? 2 : 1;
             }
