@@ -56,7 +56,8 @@ typedef enum {
     HARP_KERNEL_AUTO = 0,
     HARP_KERNEL_GENERIC = 1,   /* CUDA cores, any plan                                   */
     HARP_KERNEL_FAST = 2,      /* tensor cores, whole rows per CTA                       */
-    HARP_KERNEL_SPLIT = 3      /* tensor cores, two passes over column groups (wide rows) */
+    HARP_KERNEL_SPLIT = 3,     /* tensor cores, two passes over column groups (wide rows) */
+    HARP_KERNEL_TMEM = 4       /* tcgen05.mma, 128 rows per tile, operands in tensor memory */
 } harp_kernel_t;
 
 /* Build a processor (Eq. 6-9 of the paper; Algorithm 1 lines 2 and 7-8 for the stride
@@ -265,6 +266,13 @@ harp_status_t harp_diag_weighted_error(const void *Wt, const void *Wq, int64_t d
  *   x_host   HOST n_rows x d, overwritten with the result */
 harp_status_t harp_apply_host(harp_plan_t *plan, void *x_host, int64_t n_rows,
                               harp_dtype_t dtype, int transpose);
+
+/* Device-side wait status of the plan's HARP_KERNEL_TMEM kernels.  Every wait inside those kernels
+ * (on a bulk copy, on the tensor core, on another warp) has an iteration limit; a wait that runs out
+ * sets a device word, the kernel releases its tensor memory and returns, and the rows it was working
+ * on are left undefined.  Returns 0 if no wait has given up since the plan was built, a positive
+ * code naming the wait otherwise, -1 for NULL or a failed copy.  Synchronises with the device. */
+int32_t harp_plan_error_word(const harp_plan_t *plan);
 
 /* Number of kernels this library has launched in the calling process (all plans). */
 int64_t harp_launch_count(void);

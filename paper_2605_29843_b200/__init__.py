@@ -16,7 +16,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libharp.so")
 
 HARP_F32, HARP_BF16 = 0, 1
-KERNEL_AUTO, KERNEL_GENERIC, KERNEL_FAST, KERNEL_SPLIT = 0, 1, 2, 3
+KERNEL_AUTO, KERNEL_GENERIC, KERNEL_FAST, KERNEL_SPLIT, KERNEL_TMEM = 0, 1, 2, 3, 4
 HARP_OK = 0
 HARP_ERR_UNSUPPORTED = 8
 
@@ -81,6 +81,8 @@ def lib() -> ctypes.CDLL:
         L.harp_diag_weighted_error.argtypes = [vp, vp, i64, i64, ctypes.c_int, vp, ctypes.c_int, vp, vp]
         L.harp_apply_host.restype = ctypes.c_int
         L.harp_apply_host.argtypes = [vp, vp, i64, ctypes.c_int, ctypes.c_int]
+        L.harp_plan_error_word.restype = i32
+        L.harp_plan_error_word.argtypes = [vp]
         L.harp_launch_count.restype = i64
         L.harp_launch_count.argtypes = []
         L.harp_status_string.restype = ctypes.c_char_p
@@ -91,6 +93,10 @@ def lib() -> ctypes.CDLL:
 
 def status_string(status: int) -> str:
     return lib().harp_status_string(int(status)).decode()
+
+
+def harp_plan_error_word(plan) -> int:
+    return int(lib().harp_plan_error_word(plan.handle if hasattr(plan, "handle") else plan))
 
 
 def harp_launch_count() -> int:

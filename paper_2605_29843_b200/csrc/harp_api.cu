@@ -44,6 +44,8 @@ extern "C" const char *harp_status_string(harp_status_t s) {
     return "unknown status";
 }
 
+extern "C" int32_t harp_plan_error_word(const harp_plan_t *plan) { return plan ? harp_tm_error_word(plan) : -1; }
+
 extern "C" int64_t harp_launch_count(void) { return g_harp_launches.load(std::memory_order_relaxed); }
 
 extern "C" harp_status_t harp_plan_create(harp_plan_t **out, int64_t d, int32_t n_stages,
@@ -150,6 +152,10 @@ extern "C" harp_status_t harp_plan_create(harp_plan_t **out, int64_t d, int32_t 
         if (fs != HARP_OK && fs != HARP_ERR_UNSUPPORTED) st = fs;
     }
     if (st == HARP_OK) {
+        harp_status_t fs = harp_tm_build(p);
+        if (fs != HARP_OK && fs != HARP_ERR_UNSUPPORTED) st = fs;
+    }
+    if (st == HARP_OK) {
         harp_status_t fs = harp_col_build(p);
         if (fs != HARP_OK && fs != HARP_ERR_UNSUPPORTED) st = fs;
     }
@@ -169,6 +175,7 @@ extern "C" void harp_plan_destroy(harp_plan_t *p) {
         harp_fast_destroy(p);
         harp_split_destroy(p);
         harp_col_destroy(p);
+        harp_tm_destroy(p);
         for (int i = 0; i < harp_plan::kStages; ++i) {
             if (p->stage_stream[i]) { cudaStreamSynchronize(p->stage_stream[i]); cudaStreamDestroy(p->stage_stream[i]); }
             if (p->stage_buf[i]) cudaFree(p->stage_buf[i]);
@@ -191,7 +198,7 @@ extern "C" harp_status_t harp_apply_ex(const harp_plan_t *plan, void *x, int64_t
     if (dtype != HARP_F32 && dtype != HARP_BF16) return HARP_ERR_BAD_DTYPE;
     if (n_rows < 0) return HARP_ERR_BAD_DIM;
     if (kernel != HARP_KERNEL_AUTO && kernel != HARP_KERNEL_GENERIC && kernel != HARP_KERNEL_FAST &&
-        kernel != HARP_KERNEL_SPLIT)
+        kernel != HARP_KERNEL_SPLIT && kernel != HARP_KERNEL_TMEM)
         return HARP_ERR_UNSUPPORTED;
     if (n_rows == 0) return HARP_OK;
     if (!x) return HARP_ERR_NULL;
@@ -201,6 +208,7 @@ extern "C" harp_status_t harp_apply_ex(const harp_plan_t *plan, void *x, int64_t
     if (kernel == HARP_KERNEL_GENERIC) return harp_generic_apply(plan, x, n_rows, dtype, transpose, s);
     if (kernel == HARP_KERNEL_FAST) return harp_fast_apply(plan, x, n_rows, dtype, transpose, s);
     if (kernel == HARP_KERNEL_SPLIT) return harp_split_apply(plan, x, n_rows, dtype, transpose, s);
+    if (kernel == HARP_KERNEL_TMEM) return harp_tm_apply(plan, x, n_rows, dtype, transpose, s);
     harp_status_t st = harp_fast_apply(plan, x, n_rows, dtype, transpose, s);
     if (st != HARP_ERR_UNSUPPORTED) return st;
     st = harp_split_apply(plan, x, n_rows, dtype, transpose, s);

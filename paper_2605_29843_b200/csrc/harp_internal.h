@@ -22,6 +22,7 @@ struct StageTable {
 
 struct FastPlan;   // tensor-core path data, whole rows per CTA (harp_fast.cu)
 struct SplitPlan;  // tensor-core path data, two passes over column groups (harp_split.cu)
+struct TmPlan;    // tensor-memory path data: tcgen05.mma, rows as the M dimension (harp_tm.cu)
 struct ColPlan;    // tensor-core path data for applying the plan down the columns of a matrix (harp_col.cu)
 
 struct harp_plan {
@@ -48,6 +49,7 @@ struct harp_plan {
     FastPlan *fast = nullptr;
     SplitPlan *split = nullptr;
     ColPlan *col = nullptr;
+    TmPlan *tm = nullptr;
     // staging owned by harp_apply_host
     static constexpr int kStages = 4;
     void *stage_buf[kStages] = {nullptr, nullptr, nullptr, nullptr};
@@ -74,6 +76,13 @@ harp_status_t harp_split_build(harp_plan *plan);
 void harp_split_destroy(harp_plan *plan);
 harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype,
                                int transpose, cudaStream_t stream);
+
+// tensor-memory path (harp_tm.cu)
+harp_status_t harp_tm_build(harp_plan *plan);
+void harp_tm_destroy(harp_plan *plan);
+harp_status_t harp_tm_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype,
+                            int transpose, cudaStream_t stream);
+int32_t harp_tm_error_word(const harp_plan *plan);
 
 // column-side apply for two-sided processing (harp_col.cu): plan applied down the columns of a
 // dim(plan) x n_cols row-major matrix with leading dimension ld

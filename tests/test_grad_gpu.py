@@ -84,6 +84,48 @@ def test_accumulate_and_row_chunks_add_up():
     assert float(out.abs().max()) == 0.0
 
 
+def _rows(seed, n, d, dtype):
+    rng = np.random.default_rng(seed)
+    return host_rows(rng.standard_normal((n, d)), dtype), host_rows(rng.standard_normal((n, d)), dtype)
+
+
+def test_every_entry_at_full_dimension_cfg2():
+    """cfg2's plan (d = 4096, six radix-4 stages, digit-reversal permutation) on 4100 bf16 rows --
+    more than one internal row chunk, ragged against every slice size: every entry of every
+    stage's gradient against the oracle's chain rule through Algorithm 1."""
+    spec = wl.config(2).plans["q"]
+    plan = harp.plan_from_spec(spec)
+    oplan = orc.OraclePlan.from_spec(spec)
+    xh, gh = _rows(90, 4100, spec.d, "bf16")
+    got, _, _ = _gpu_grad(plan, xh, gh, "bf16")
+    want = _flat(orc.grad_blocks(oplan, promote(xh, "bf16"), promote(gh, "bf16")))
+    assert got.shape == want.shape
+    off = 0
+    for t, b in enumerate(spec.radices):                     # per stage, so a quiet stage cannot hide
+        n = spec.d * b
+        g, w = got[off:off + n], want[off:off + n]
+        off += n
+        assert np.max(np.abs(g - w)) <= 2e-5 * np.max(np.abs(w)), t
+
+
+def test_every_entry_at_full_dimension_cfg4():
+    """cfg4's plan (d = 14336, radices 16, 16, 8, 7): all entries on 256 rows, and again on a batch
+    long enough to cross the internal row chunk."""
+    spec = list(wl.config(4).plans.values())[0]
+    plan = harp.plan_from_spec(spec)
+    oplan = orc.OraclePlan.from_spec(spec)
+    for seed, n in ((91, 256), (92, 1203)):
+        xh, gh = _rows(seed, n, spec.d, "bf16")
+        got, _, _ = _gpu_grad(plan, xh, gh, "bf16")
+        want = _flat(orc.grad_blocks(oplan, promote(xh, "bf16"), promote(gh, "bf16")))
+        off = 0
+        for t, b in enumerate(spec.radices):
+            m = spec.d * b
+            g, w = got[off:off + m], want[off:off + m]
+            off += m
+            assert np.max(np.abs(g - w)) <= 2e-5 * np.max(np.abs(w)), (n, t)
+
+
 def test_euler_identity_at_full_dimension():
     """cfg2's plan (d = 4096, six radix-4 stages, digit-reversal permutation): y is homogeneous of
     degree one in the kernels of every stage, so <K_t, dL/dK_t> = sum(y * G) for each t; y comes
