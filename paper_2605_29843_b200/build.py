@@ -34,6 +34,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-I", os.path.join(ROOT, "include"), "-I", os.path.join(HERE, "csrc")]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    if os.environ.get("HARP_TM_TIMING"):          # per-section cycle counters in the tensor-memory kernels
+        cmd += ["-DHARP_TM_TIMING"]
     cmd += sources() + ["-o", LIB]
     subprocess.check_call(cmd)
     return LIB

@@ -39,6 +39,7 @@
 #include "harp_internal.h"
 #include "harp_mma.cuh"
 #include "harp_fuse.h"
+#include "harp_tm_ptx.cuh"
 
 namespace {
 
@@ -74,8 +75,26 @@ struct FastParams {
     // offset of every 8-coordinate chunk of a row) and the per-phase item tables
     const int32_t *tables;
     int32_t tables_len;
+    // phases whose block fragments a CTA keeps in tensor memory for all its tiles (bit p = phase p):
+    // warp w reads the fragments of its own items w and w + 16 from its 32 lanes, 32 columns per item
+    uint32_t tm_mask;
     PhaseDesc ph[kMaxPhases];
 };
+
+// fragments of one item (eight blocks, one uint4 per lane and block): from tensor memory when the
+// phase is kept there, else from global memory
+__device__ __forceinline__ void load_frag8(uint4 (&bf)[8], const uint4 *bp, bool in_tm, uint32_t tm_addr) {
+    if (in_tm) {
+        uint32_t v[32];
+        harp_tm::tmem_ld32(tm_addr, v);
+        harp_tm::tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 8; ++e) bf[e] = make_uint4(v[4 * e], v[4 * e + 1], v[4 * e + 2], v[4 * e + 3]);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) bf[e] = __ldg(bp + e * 32);
+    }
+}
 
 // ----------------------------------------------------------------------------- device
 
@@ -85,15 +104,20 @@ struct TileCtx {
     int pitch, lane, warp, g, q;
     __nv_bfloat16 *xA, *xB;  // global rows g and g+8 of the tile (clamped to the batch)
     bool okA, okB;
+    uint32_t tm_warp;        // tensor-memory address of this warp's fragment columns
 };
+// tensor-memory address of item `it` of the phase kept in slot `slot` (0 or 1), for the calling warp
+__device__ __forceinline__ uint32_t tm_item(const TileCtx &c, int slot, int it) {
+    return c.tm_warp + (uint32_t)((slot * 2 + (it >> 4)) * 32);
+}
 
 // ---- MODE_SS, B = 16: load / store of one item's operands
-__device__ __forceinline__ void ss16_load(const TileCtx &c, const PhaseDesc &ph, int it, uint4 (&raw)[4][2], uint4 (&bf)[8]) {
+__device__ __forceinline__ void ss16_load(const TileCtx &c, const PhaseDesc &ph, int it, uint4 (&raw)[4][2], uint4 (&bf)[8],
+                                          int tm_slot) {
     const uint32_t a0 = c.sbase + 2u * (uint32_t)(c.g * c.pitch + c.q * ph.lane_step + c.tab[ph.items_off + it]);
     const uint32_t a1 = a0 + 2u * (uint32_t)(8 * c.pitch);
     const uint4 *bp = ph.bfrag + (size_t)it * 256 + c.lane;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) bf[e] = __ldg(bp + e * 32);
+    load_frag8(bf, bp, tm_slot >= 0, tm_item(c, tm_slot, it));
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         raw[j][0] = lds128(a0 + 2u * ph.j_off[j]);
@@ -110,7 +134,8 @@ __device__ __forceinline__ void ss16_store(const TileCtx &c, const PhaseDesc &ph
     }
 }
 // ---- MODE_GS: operands from global memory
-__device__ __forceinline__ void gs_load(const TileCtx &c, const PhaseDesc &ph, int it, uint4 (&raw)[4][2], uint4 (&bf)[8]) {
+__device__ __forceinline__ void gs_load(const TileCtx &c, const PhaseDesc &ph, int it, uint4 (&raw)[4][2], uint4 (&bf)[8],
+                                        int tm_slot) {
     const int32_t *tab = c.tab + ph.items_off + it * 24;
     const uint4 *bp = ph.bfrag + (size_t)it * 256 + c.lane;
 #pragma unroll
@@ -119,8 +144,7 @@ __device__ __forceinline__ void gs_load(const TileCtx &c, const PhaseDesc &ph, i
         raw[j][0] = ldg128_stream(c.xA + off);
         raw[j][1] = ldg128_stream(c.xB + off);
     }
-#pragma unroll
-    for (int e = 0; e < 8; ++e) bf[e] = __ldg(bp + e * 32);
+    load_frag8(bf, bp, tm_slot >= 0, tm_item(c, tm_slot, it));
 }
 __device__ __forceinline__ void gs_store(const TileCtx &c, const PhaseDesc &ph, int it, const uint32_t (&mats)[8][4]) {
     const int32_t *tab = c.tab + ph.items_off + it * 24 + 16;
@@ -153,7 +177,33 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
     int32_t *tab_s = reinterpret_cast<int32_t *>(smem_raw + (size_t)kTileRows * pitch * 2);
     for (int i = threadIdx.x; i < P.tables_len; i += NT) tab_s[i] = __ldg(P.tables + i);
     c.tab = tab_s;
+    // ---- block fragments of up to two phases into tensor memory, once per CTA ----
+    uint32_t &tm_base_s = *reinterpret_cast<uint32_t *>(tab_s + P.tables_len);   // one word after the tables
+    if (P.tm_mask) {
+        if (c.warp == 0) harp_tm::tmem_alloc(smem_u32(&tm_base_s), 512);
+        harp_tm::tc_fence_before();
+    }
     __syncthreads();
+    c.tm_warp = 0;
+    if (P.tm_mask) {
+        harp_tm::tc_fence_after();
+        c.tm_warp = tm_base_s + ((uint32_t)((c.warp & 3) * 32) << 16) + (uint32_t)((c.warp >> 2) * 128);
+        int slot = 0;
+        for (int p = 0; p < P.n_phases; ++p) {
+            if (!((P.tm_mask >> p) & 1u)) continue;
+            for (int it = c.warp; it < P.ph[p].n_items; it += NW) {
+                uint32_t v[32];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const uint4 f = __ldg(P.ph[p].bfrag + (size_t)it * 256 + e * 32 + c.lane);
+                    v[4 * e] = f.x; v[4 * e + 1] = f.y; v[4 * e + 2] = f.z; v[4 * e + 3] = f.w;
+                }
+                harp_tm::tmem_st32(tm_item(c, slot, it), v);
+            }
+            ++slot;
+        }
+        harp_tm::tmem_wait_st();
+    }
     const int warp = c.warp, lane = c.lane;
 
     // All CTAs have the same work, so without this they copy their tiles in step and share the
@@ -192,6 +242,7 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
         for (int p = 0; p < P.n_phases; ++p) {
             const PhaseDesc &ph = P.ph[p];
             const int n = ph.n_items;
+            const int tm_slot = ((P.tm_mask >> p) & 1u) ? __popc(P.tm_mask & ((1u << p) - 1u)) : -1;
             if ((MODES & bit(MODE_CC)) && ph.mode == MODE_CC) {
                 // lane -> (matrix row, 8-column half) of the 16x16 (or 16x8) operand tile
                 const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
@@ -228,7 +279,7 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
                 uint4 raw[4][2], bf[8];
                 uint32_t unused[8][4];
                 for (int it = warp; it < n; it += NW) {
-                    ss16_load(c, ph, it, raw, bf);
+                    ss16_load(c, ph, it, raw, bf, tm_slot);
                     octet_mma16<true>(raw, bf, unused);
                     ss16_store(c, ph, it, raw);
                 }
@@ -257,7 +308,7 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
                 uint4 raw[4][2], bf[8];
                 uint32_t mats[8][4];
                 for (int it = warp; it < n; it += NW) {
-                    gs_load(c, ph, it, raw, bf);
+                    gs_load(c, ph, it, raw, bf, tm_slot);
                     octet_mma16<false>(raw, bf, mats);
                     gs_store(c, ph, it, mats);
                 }
@@ -268,8 +319,7 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
                 for (int it = warp; it < n; it += NW) {
                     const int32_t *tab = tab_s + ph.items_off + it * 24;
                     uint4 bf[8], out[4][2];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) bf[e] = __ldg(ph.bfrag + (size_t)it * 256 + e * 32 + lane);
+                    load_frag8(bf, ph.bfrag + (size_t)it * 256 + lane, tm_slot >= 0, tm_item(c, tm_slot, it));
 #pragma unroll
                     for (int w = 0; w < 4; ++w) {
                         float acc[2][2][4];
@@ -303,8 +353,7 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
                 for (int it = warp; it < n; it += NW) {
                     const int32_t *tab = tab_s + ph.items_off + it * 24;
                     uint4 bf[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) bf[e] = __ldg(ph.bfrag + (size_t)it * 256 + e * 32 + lane);
+                    load_frag8(bf, ph.bfrag + (size_t)it * 256 + lane, tm_slot >= 0, tm_item(c, tm_slot, it));
                     uint4 out[4][2];
 #pragma unroll
                     for (int w = 0; w < 4; ++w) {
@@ -348,6 +397,11 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
             }
             __syncthreads();
         }
+    }
+    if (P.tm_mask) {
+        harp_tm::tc_fence_before();
+        __syncthreads();
+        if (c.warp == 0) harp_tm::tmem_dealloc(tm_base_s, 512);
     }
 }
 
@@ -902,9 +956,20 @@ harp_status_t harp_fast_build(harp_plan *plan) {
             }
             D.bfrag = reinterpret_cast<const uint4 *>(upload(fp, frag, st));
         }
+        // up to two phases whose items come eight blocks at a time keep their fragments in tensor memory
+        // (2 x 32 items x 4 KB fill its 256 KB)
+        P.tm_mask = 0;
+        if (!getenv("HARP_FAST_NO_TMEM")) {
+            int kept = 0;
+            for (int k = 0; k < np && kept < 2; ++k) {
+                const PhaseDesc &D = P.ph[k];
+                const bool eight = D.B == 16 && (D.mode == MODE_SS || D.mode == MODE_GS || D.mode == MODE_PO || D.mode == MODE_CG);
+                if (eight && D.n_items <= 2 * (kThreads / 32)) { P.tm_mask |= 1u << k; ++kept; }
+            }
+        }
         P.tables = upload(fp, tables, st);
         P.tables_len = (int32_t)tables.size();
-        fp->smem_bytes = std::max(fp->smem_bytes, tile_bytes + tables.size() * sizeof(int32_t));
+        fp->smem_bytes = std::max(fp->smem_bytes, tile_bytes + tables.size() * sizeof(int32_t) + 16);
     }
     if (st == HARP_OK && fp->smem_bytes > 227u * 1024u) st = HARP_ERR_UNSUPPORTED;
     if (st == HARP_OK) {

@@ -78,6 +78,20 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
     asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 
+// Per-section cycle counters (build with -DHARP_TM_TIMING): summed over CTAs by one thread per role.
+//  0 tiles | producer: 1 wait for a free buffer, 2 issue | MMA: 3 wait for A, 4 issue
+//  store: 5 wait for a finished tile, 6 wait for the store to have read it
+//  epilogue (row 0 of warpgroup 0): 7 wait for the tile, 8 row -> A, 9 wait for D (phase 1), 10 D -> A (between
+//  the phases), 11 wait for D (phase 2), 12 D -> tile buffer
+__device__ long long g_tm_timing[16];
+#ifdef HARP_TM_TIMING
+#define TM_T(var) const long long var = clock64()
+#define TM_ACC(slot, a, b) acc[slot] += (b) - (a)
+#else
+#define TM_T(var)
+#define TM_ACC(slot, a, b)
+#endif
+
 struct Waiter {
     volatile int *dead;
     int32_t *err;
@@ -163,11 +177,15 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
         if (lane == 0) {
             int cur_col = -1, slot = 1;
             int64_t issued = 0;
+            long long acc[16] = {0};
             for (int64_t t = t_begin; t < t_end; ++t) {
                 const int64_t i = t - t_begin;
                 const int b = (int)(i % kNBuf);
                 const uint32_t par = (uint32_t)((i / kNBuf) & 1);
+                TM_T(c0);
                 if (!wait(bar_empty + 8 * b, par ^ 1, 1)) break;
+                TM_T(c1);
+                TM_ACC(1, c0, c1);
                 const int col = (int)(t / P.n_row_tiles), row0 = (int)(t % P.n_row_tiles) * kRows;
                 uint32_t bytes = kTileBytes;
                 const bool new_frag = col != cur_col;
@@ -191,7 +209,14 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
                     tma_load_3d(dst, &tmap, lo * 16, row0, hi * 16, bar_full + 8 * b);
                 }
                 issued = i + 1;
+                TM_T(c2);
+                TM_ACC(2, c1, c2);
             }
+#ifdef HARP_TM_TIMING
+            atomicAdd((unsigned long long *)&g_tm_timing[0], (unsigned long long)(t_end > t_begin ? t_end - t_begin : 0));
+            atomicAdd((unsigned long long *)&g_tm_timing[1], (unsigned long long)acc[1]);
+            atomicAdd((unsigned long long *)&g_tm_timing[2], (unsigned long long)acc[2]);
+#endif
             if (dead_s) {
                 // leave no copy in flight: bounded wait for the loads issued last
                 for (int64_t k = issued > kNBuf ? issued - kNBuf : 0; k < issued; ++k)
@@ -205,13 +230,17 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
             const uint32_t idesc = instr_desc(128, 16);
             int cur_col = -1, slot = 1;
             uint32_t ua = 0;
+            long long acc[16] = {0};
             for (int64_t t = t_begin; t < t_end; ++t) {
                 const int col = (int)(t / P.n_row_tiles);
                 if (col != cur_col) { cur_col = col; slot ^= 1; }
                 bool ok = true;
 #pragma unroll
                 for (int ph = 0; ph < NPH; ++ph) {
+                    TM_T(c0);
                     if (!wait(bar_a, ua & 1, 3)) { ok = false; break; }
+                    TM_T(c1);
+                    TM_ACC(3, c0, c1);
                     ++ua;
                     tc_fence_after();
                     const uint32_t a_col = ph == 0 ? kColA1 : kColA2;
@@ -225,17 +254,27 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
                         }
                         mma_commit(bar_d + 8 * g);
                     }
+                    TM_T(c2);
+                    TM_ACC(4, c1, c2);
                 }
                 if (!ok) break;
             }
+#ifdef HARP_TM_TIMING
+            atomicAdd((unsigned long long *)&g_tm_timing[3], (unsigned long long)acc[3]);
+            atomicAdd((unsigned long long *)&g_tm_timing[4], (unsigned long long)acc[4]);
+#endif
         }
     } else if (warp == 2) {
         // ---------------- store: finished tiles back to global memory ----------------
         if (lane == 0) {
+            long long acc[16] = {0};
             for (int64_t t = t_begin; t < t_end; ++t) {
                 const int64_t i = t - t_begin;
                 const int b = (int)(i % kNBuf);
+                TM_T(c0);
                 if (!wait(bar_out + 8 * b, (uint32_t)((i / kNBuf) & 1), 4)) break;
+                TM_T(c1);
+                TM_ACC(5, c0, c1);
                 const int col = (int)(t / P.n_row_tiles), row0 = (int)(t % P.n_row_tiles) * kRows;
                 const uint32_t src = buf0 + b * kTileBytes;
                 if (FMT == FMT_C) {
@@ -248,8 +287,14 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
                 bulk_commit();
                 bulk_wait_read0();
                 mbar_arrive(bar_empty + 8 * b);
+                TM_T(c2);
+                TM_ACC(6, c1, c2);
             }
             bulk_wait0();
+#ifdef HARP_TM_TIMING
+            atomicAdd((unsigned long long *)&g_tm_timing[5], (unsigned long long)acc[5]);
+            atomicAdd((unsigned long long *)&g_tm_timing[6], (unsigned long long)acc[6]);
+#endif
         }
     } else if (warp >= 4) {
         // ---------------- epilogue warpgroups: thread = row = lane of tensor memory ----------------
@@ -257,11 +302,15 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
         const int r = ((warp & 3) << 5) | lane;             // row of the tile
         const uint32_t tlane = tmem + ((uint32_t)((warp & 3) << 5) << 16);
         uint32_t ud = 0;
+        long long acc[16] = {0};
         for (int64_t t = t_begin; t < t_end; ++t) {
             const int64_t i = t - t_begin;
             const int b = (int)(i % kNBuf);
             const uint32_t buf = buf0 + b * kTileBytes;
+            TM_T(e0);
             if (!wait(bar_full + 8 * b, (uint32_t)((i / kNBuf) & 1), 5)) break;
+            TM_T(e1);
+            TM_ACC(7, e0, e1);
             // --- row from shared memory to the A operand of the first phase ---
             {
                 uint32_t a[64];
@@ -294,9 +343,13 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar_a);
+            TM_T(e2);
+            TM_ACC(8, e1, e2);
             if (!wait(bar_d + 8 * g, ud & 1, 6)) break;
             ++ud;
             tc_fence_after();
+            TM_T(e3);
+            TM_ACC(9, e2, e3);
             if (NPH == 2) {
                 // --- between the phases: D (fp32) -> A of the other index (bf16 pairs over neighbouring blocks) ---
                 uint32_t p[64];
@@ -309,10 +362,15 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
                 tmem_wait_st();
                 tc_fence_before();
                 mbar_arrive(bar_a);
+                TM_T(e4);
+                TM_ACC(10, e3, e4);
                 if (!wait(bar_d + 8 * g, ud & 1, 7)) break;
                 ++ud;
                 tc_fence_after();
+                TM_T(e5);
+                TM_ACC(11, e4, e5);
             }
+            TM_T(e6);
             // --- result back into the tile buffer (in place), rounded once to bf16 ---
             if (CROSS_OUT) {
                 uint32_t p[64];
@@ -342,7 +400,13 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
             tc_fence_before();
             fence_async_smem();
             mbar_arrive(bar_out + 8 * b);
+            TM_T(e7);
+            TM_ACC(12, e6, e7);
         }
+#ifdef HARP_TM_TIMING
+        if (warp == 4 && lane == 0)
+            for (int k = 7; k <= 12; ++k) atomicAdd((unsigned long long *)&g_tm_timing[k], (unsigned long long)acc[k]);
+#endif
     }
     __syncwarp();
     tc_fence_before();
@@ -627,6 +691,18 @@ harp_status_t harp_tm_apply(const harp_plan *plan, void *x, int64_t n_rows, harp
         g_harp_launches.fetch_add(1, std::memory_order_relaxed);
     }
     return HARP_OK;
+}
+
+// Copies the per-section cycle counters to out[16] (zeros unless built with -DHARP_TM_TIMING) and
+// clears them if asked.
+extern "C" int32_t harp_debug_tm_timing(int64_t *out, int32_t reset) {
+    if (!out) return -1;
+    if (cudaMemcpyFromSymbol(out, g_tm_timing, sizeof(long long) * 16) != cudaSuccess) return -1;
+    if (reset) {
+        const long long zero[16] = {0};
+        if (cudaMemcpyToSymbol(g_tm_timing, zero, sizeof(zero)) != cudaSuccess) return -1;
+    }
+    return 0;
 }
 
 // Non-zero if a kernel of this plan's tensor-memory path gave up on a wait since the plan was built
