@@ -63,7 +63,9 @@ typedef enum {
 /* Build a processor (Eq. 6-9 of the paper; Algorithm 1 lines 2 and 7-8 for the stride
  * and block-kernel layout).
  *   out      HOST  receives the plan; untouched on error
- *   d        transformed dimension, 2 <= d <= 2^20
+ *   d        transformed dimension, 2 <= d <= 2^20 (plans are built for any such d; whether a kernel
+ *            exists for it is decided per call: fp32 or permuted rows beyond d = 32768 and bf16 rows
+ *            no tensor-core path takes return HARP_ERR_UNSUPPORTED from harp_apply)
  *   n_stages m >= 1;  radices HOST int32[m], each >= 2, product == d
  *   perm     HOST int32[d] bijection, forward gathers v[i] = u[perm[i]]; NULL = identity
  *   signs    HOST int8[d] with entries +1/-1;  NULL = all +1
@@ -101,6 +103,18 @@ harp_status_t harp_blocks_from_theta(int32_t b, int64_t n_blocks, const float *t
                                      const int8_t *theta_q, const float *scales,
                                      const float *mixer, float *out_blocks);
 
+/* The same reconstruction on the GPU (Section "Parameter quantization for deployment", appendix "Int8
+ * storage of HARP parameters": the orthogonal block is rebuilt from the stored angles / upper triangle
+ * at runtime).  Every pointer is DEVICE memory on the current device, with the layouts of
+ * harp_blocks_from_theta; one thread block per matrix block solves (I + A) Q = I - A in fp64 (Gauss-
+ * Jordan with partial pivoting in shared memory) and multiplies by the mixer, one rounding to fp32.
+ * b <= harp_theta_device_max_radix() (54), else HARP_ERR_UNSUPPORTED.  Asynchronous on stream;
+ * allocates nothing. */
+harp_status_t harp_blocks_from_theta_device(int32_t b, int64_t n_blocks, const float *theta,
+                                            const int8_t *theta_q, const float *scales,
+                                            const float *mixer, float *out_blocks, void *stream);
+int32_t harp_theta_device_max_radix(void);
+
 /* Gradient with respect to the stored parameters of one stage, given the gradient with respect to
  * its block kernels (harp_grad_blocks, copied to the host): the chain rule through B_c = Q(theta_c) G_b
  * (Eq. 9-11), i.e. what the parameter update of Algorithm 3 needs.  All pointers HOST; no CUDA call.
@@ -112,7 +126,8 @@ harp_status_t harp_blocks_from_theta(int32_t b, int64_t n_blocks, const float *t
 harp_status_t harp_grad_theta(int32_t b, int64_t n_blocks, const float *theta, const float *mixer,
                               const float *grad_blocks, float *grad_theta);
 
-/* harp_plan_create with every stage's blocks rebuilt by harp_blocks_from_theta.  theta, theta_q,
+/* harp_plan_create with every stage's blocks rebuilt from the stored parameters: by the device
+ * kernels of harp_blocks_from_theta_device for radices they take, by harp_blocks_from_theta otherwise.  theta, theta_q,
  * scales, mixers are HOST arrays of n_stages pointers (theta or theta_q may be NULL as a whole;
  * mixers may be NULL if every radix is a power of two). */
 harp_status_t harp_plan_create_from_theta(harp_plan_t **out, int64_t d, int32_t n_stages,
@@ -146,7 +161,15 @@ int64_t harp_plan_dim(const harp_plan_t *plan);
  *   x        DEVICE n_rows x d, dtype fp32 or bf16, overwritten with the result
  *   stream   a cudaStream_t passed as void* (NULL = default stream)
  * Asynchronous on stream; does not synchronise.  n_rows == 0 returns HARP_OK without
- * a launch.  bf16 results are rounded once, to nearest even, at the store. */
+ * a launch.  A plan may be applied from several streams at once.
+ * Arithmetic.  fp32 rows: fp32 block kernels, fp32 accumulate, the result is the fp32 sum (one
+ * rounding per stage).  bf16 rows on the tensor-core kernels (what HARP_KERNEL_AUTO picks for
+ * bf16 whenever a plan has one): neighbouring stages are fused at plan time into dense blocks of
+ * width 8 to 64 (fp64 product, rounded once to bf16), every block product accumulates in fp32,
+ * and the rows are rounded to bf16, to nearest even, after every fused group of stages -- two to
+ * five roundings per coordinate instead of one, measured 2e-4 to 7e-4 of the row norm against a
+ * tolerance of 8e-3.  bf16 rows on HARP_KERNEL_GENERIC: fp32 throughout, one rounding at the
+ * store. */
 harp_status_t harp_apply(const harp_plan_t *plan, void *x, int64_t n_rows, harp_dtype_t dtype,
                          int transpose, void *stream);
 
@@ -173,7 +196,10 @@ harp_status_t harp_apply_passes(const harp_plan_t *const *plans, int32_t n_passe
  *   W        DEVICE d_out x d_in row-major, d_out = dim(plan_out), d_in = dim(plan_in)
  *   scratch  DEVICE buffer of harp_two_sided_scratch_bytes(...) bytes, 256-byte aligned,
  *            or NULL to let the call allocate and free it on the stream
- *            (cudaMallocAsync/cudaFreeAsync).
+ *            (cudaMallocAsync/cudaFreeAsync).  It is used only when the column side has to go
+ *            through a transposed copy of W (plan_out with a permutation, fp32, or d_in not a
+ *            multiple of 8); otherwise the columns are processed in place and it is ignored.
+ * Both plans must live on the current device (else HARP_ERR_DIM_MISMATCH).
  * Asynchronous on stream. */
 harp_status_t harp_apply_two_sided(void *W, harp_dtype_t dtype, const harp_plan_t *plan_out,
                                    const harp_plan_t *plan_in, void *scratch, void *stream);
@@ -186,10 +212,13 @@ int64_t harp_two_sided_scratch_bytes(const harp_plan_t *plan_out, const harp_pla
  * point exists for deployment, not for the method).  It is meant for callers that cannot
  * allocate device memory at call time -- a serving process whose memory pool was sized
  * once at start-up, a host framework that owns the whole device budget, or any context in
- * which an allocation would synchronise or fail.  It computes exactly what
- * harp_apply_two_sided computes, but keeps the transposed copy of W in a fixed array that
- * is compiled into the library; every device that loads the library holds that array
- * (harp_two_sided_static_capacity_bytes() = 32 MiB) until the process exits.
+ * which an allocation would synchronise or fail.  It computes the same map as
+ * harp_apply_two_sided, always by the transpose route (rows through Q_in, transpose, rows
+ * through Q_out, transpose back; bf16 results can differ from the other entry point's in the
+ * last rounding, and it costs two more passes over W than the in-place column kernels), and
+ * keeps the transposed copy of W in a fixed array that is compiled into the library; the array
+ * becomes resident when the library's module is loaded on a device (at the latest by the first
+ * call) and stays (harp_two_sided_static_capacity_bytes() = 32 MiB) until the process exits.
  *   W        DEVICE d_out x d_in row-major, overwritten; d_out*d_in*sizeof(dtype) must not
  *            exceed the capacity, otherwise HARP_ERR_TOO_LARGE and nothing is launched
  *   plans    must live on the current device (else HARP_ERR_DIM_MISMATCH)
@@ -258,7 +287,9 @@ harp_status_t harp_diag_weighted_error(const void *Wt, const void *Wq, int64_t d
                                        harp_dtype_t dtype, const void *H, harp_dtype_t h_dtype,
                                        double *out, void *stream);
 
-/* Apply to rows that live in HOST memory (pinned memory gives full copy speed):
+/* Apply to rows that live in HOST memory (pinned memory gives full copy speed).  Unlike
+ * harp_apply this call changes the plan (its staging buffers and streams): one call at a time
+ * per plan, from one host thread.  It
  * copies chunks of 16 MiB host->device, applies, copies back, on four internal streams so
  * that copies in both directions overlap each other and the kernels; returns after the last
  * copy has completed.  The device staging buffers (four) belong to the plan and are created at

@@ -81,6 +81,10 @@ def lib() -> ctypes.CDLL:
         L.harp_diag_weighted_error.argtypes = [vp, vp, i64, i64, ctypes.c_int, vp, ctypes.c_int, vp, vp]
         L.harp_apply_host.restype = ctypes.c_int
         L.harp_apply_host.argtypes = [vp, vp, i64, ctypes.c_int, ctypes.c_int]
+        L.harp_blocks_from_theta_device.restype = ctypes.c_int
+        L.harp_blocks_from_theta_device.argtypes = [i32, i64, vp, vp, vp, vp, vp, vp]
+        L.harp_theta_device_max_radix.restype = i32
+        L.harp_theta_device_max_radix.argtypes = []
         L.harp_plan_error_word.restype = i32
         L.harp_plan_error_word.argtypes = [vp]
         L.harp_launch_count.restype = i64
@@ -193,6 +197,19 @@ def harp_grad_theta(b: int, theta, grad_blocks, mixer=None) -> np.ndarray:
     if st != HARP_OK:
         raise HarpError(st, "harp_grad_theta")
     return out
+
+
+def harp_theta_device_max_radix() -> int:
+    return int(lib().harp_theta_device_max_radix())
+
+
+def harp_blocks_from_theta_device(b: int, n_blocks: int, theta_ptr: int, theta_q_ptr: int, scales_ptr: int, mixer_ptr: int,
+                                  out_ptr: int, stream: int = 0) -> None:
+    """Device pointers in, block kernels float[n_blocks][b][b] out (device)."""
+    st = lib().harp_blocks_from_theta_device(int(b), int(n_blocks), theta_ptr or None, theta_q_ptr or None,
+                                             scales_ptr or None, mixer_ptr or None, out_ptr, stream or None)
+    if st != HARP_OK:
+        raise HarpError(st, "harp_blocks_from_theta_device")
 
 
 def harp_plan_create_from_theta(d: int, radices: Sequence[int], perm=None, signs=None, theta=None, theta_q=None,

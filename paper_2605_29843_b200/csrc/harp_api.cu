@@ -79,6 +79,7 @@ extern "C" harp_status_t harp_plan_create(harp_plan_t **out, int64_t d, int32_t 
     harp_plan *p = new (std::nothrow) harp_plan();
     if (!p) return HARP_ERR_ALLOC;
     p->d = d;
+    p->opt_no_rowvec = getenv("HARP_NO_ROWVEC") != nullptr;
     p->st.m = n_stages;
     int64_t s = 1, off = 0;
     for (int t = 0; t < n_stages; ++t) {
@@ -254,6 +255,9 @@ extern "C" harp_status_t harp_apply_two_sided(void *W, harp_dtype_t dtype, const
     if (scratch && (reinterpret_cast<uintptr_t>(scratch) & 255u) != 0) return HARP_ERR_BAD_DIM;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int64_t d_out = plan_out->d, d_in = plan_in->d;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return HARP_ERR_CUDA;
+    if (dev != plan_out->device || dev != plan_in->device) return HARP_ERR_DIM_MISMATCH;
     // row side: every row of W through Q_in
     harp_status_t st = harp_apply(plan_in, W, d_out, dtype, 0, s);
     if (st != HARP_OK) return st;
@@ -287,8 +291,8 @@ extern "C" harp_status_t harp_apply_host(harp_plan_t *plan, void *x_host, int64_
     if (!g.ok) return HARP_ERR_CUDA;
     const int64_t row_bytes = plan->d * (int64_t)harp_dtype_size(dtype);
     // staging bytes per buffer: small enough that the first copy in and the last copy out, which
-    // nothing overlaps, are a small part of the transfer; HARP_STAGE_MB overrides (for tuning)
-    const int64_t want = (int64_t)(getenv("HARP_STAGE_MB") ? std::max(1, atoi(getenv("HARP_STAGE_MB"))) : 16) << 20;
+    // nothing overlaps, are a small part of the transfer
+    const int64_t want = (int64_t)16 << 20;
     int64_t chunk_rows = std::max<int64_t>(1, want / row_bytes);
     const int64_t need = chunk_rows * row_bytes;
     if (plan->stage_bytes < need) {

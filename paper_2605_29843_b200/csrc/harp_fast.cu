@@ -959,7 +959,7 @@ harp_status_t harp_fast_build(harp_plan *plan) {
         // up to two phases whose items come eight blocks at a time keep their fragments in tensor memory
         // (2 x 32 items x 4 KB fill its 256 KB)
         P.tm_mask = 0;
-        if (!getenv("HARP_FAST_NO_TMEM")) {
+        {
             int kept = 0;
             for (int k = 0; k < np && kept < 2; ++k) {
                 const PhaseDesc &D = P.ph[k];

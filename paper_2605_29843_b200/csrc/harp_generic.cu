@@ -562,8 +562,7 @@ harp_status_t harp_generic_apply(const harp_plan *plan, void *x, int64_t n_rows,
     int max_radix = 0;
     for (int t = 0; t < bst.m; ++t) max_radix = std::max(max_radix, (int)bst.b[t]);
     if (max_radix <= 8 && !bblk) return HARP_ERR_UNSUPPORTED;
-    // HARP_NO_ROWVEC=1 forces the row-major tile (for tests of that layout)
-    const bool rowvec = d % 32 == 0 && d * 16 <= 226 * 1024 && !getenv("HARP_NO_ROWVEC");
+    const bool rowvec = d % 32 == 0 && d * 16 <= 226 * 1024 && !plan->opt_no_rowvec;
     if (rowvec && max_radix <= 4) {
         return dtype == HARP_F32 ? launch_rowvec<float, 512, false>(plan, bst, bblk, x, n_rows, transpose, stream)
                                  : launch_rowvec<__nv_bfloat16, 512, false>(plan, bst, bblk, x, n_rows, transpose, stream);

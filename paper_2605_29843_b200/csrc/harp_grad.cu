@@ -512,7 +512,8 @@ void launch_bwd_owner(int b, const float *v, const float *g, float *g_out, int64
 template <typename T>
 void launch_load(const T *x, const T *gy, int64_t rows, int64_t d, const harp_plan_t *plan, float *v0, float *g, cudaStream_t st) {
     const size_t smem = (size_t)(d + 2 * (d >> 6) + 2) * sizeof(T);
-    static const bool big_ok =
+    // per call: the attribute belongs to the current device's copy of the kernel
+    const bool big_ok = smem > 48 * 1024 &&
         cudaFuncSetAttribute(load_rows_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) == cudaSuccess;
     if (plan->d_perm && (smem <= 48 * 1024 || (big_ok && smem <= 200 * 1024)))
         launch_dep(load_rows_kernel<T>, dim3((unsigned)std::min<int64_t>(rows, 148 * 8)), dim3(kThreads), smem, st, x, gy, rows, d,
@@ -529,6 +530,11 @@ extern "C" harp_status_t harp_grad_blocks(const harp_plan_t *plan, const void *x
                                           harp_dtype_t dtype, float *grad, int accumulate, void *stream) {
     if (!plan || !grad) return HARP_ERR_NULL;
     if (dtype != HARP_F32 && dtype != HARP_BF16) return HARP_ERR_BAD_DTYPE;
+    {
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess) return HARP_ERR_CUDA;
+        if (dev != plan->device) return HARP_ERR_DIM_MISMATCH;      // the scratch pool and the plan's tables live on plan->device
+    }
     if (n_rows < 0) return HARP_ERR_BAD_DIM;
     if (n_rows > 0 && (!x || !gy)) return HARP_ERR_NULL;
     const size_t es = harp_dtype_size(dtype);

@@ -50,6 +50,9 @@ struct harp_plan {
     SplitPlan *split = nullptr;
     ColPlan *col = nullptr;
     TmPlan *tm = nullptr;
+    // test-only switch, read from the environment once, when the plan is built (HARP_NO_ROWVEC=1: the
+    // CUDA-core kernels keep their tile row-major)
+    bool opt_no_rowvec = false;
     // staging owned by harp_apply_host
     static constexpr int kStages = 4;
     void *stage_buf[kStages] = {nullptr, nullptr, nullptr, nullptr};

@@ -1,6 +1,7 @@
 // Plan-side helpers of the C ABI (host code): the greedy Mixed-Radix schedule, block kernels
 // rebuilt from stored parameters (Givens angle / Cayley upper triangle, optionally int8 with a
 // per-block scale), and the Kronecker fallback written as an ordinary stage list.
+#include <algorithm>
 #include <cmath>
 #include <new>
 #include <vector>
@@ -183,6 +184,42 @@ extern "C" harp_status_t harp_grad_theta(int32_t b, int64_t n_blocks, const floa
     return HARP_OK;
 }
 
+namespace {
+
+// One stage's block kernels through the device kernels: parameters up, blocks rebuilt on the GPU,
+// blocks back (the plan builder fuses stages on the host).  HARP_ERR_UNSUPPORTED for radices the
+// device kernels do not take.
+harp_status_t stage_blocks_on_device(int b, int64_t n_blocks, const float *theta, const int8_t *theta_q, const float *scales,
+                                     const float *mixer, float *out_host) {
+    if (b > harp_theta_device_max_radix()) return HARP_ERR_UNSUPPORTED;
+    if ((!theta && !theta_q) || (theta_q && !theta && !scales)) return HARP_ERR_NULL;
+    if (!mixer && !is_pow2(b)) return HARP_ERR_NULL;
+    const int np = harp_theta_params_per_block(b);
+    void *d_theta = nullptr, *d_scales = nullptr, *d_mixer = nullptr, *d_out = nullptr;
+    const size_t theta_bytes = (size_t)n_blocks * np * (theta ? sizeof(float) : 1);
+    harp_status_t st = HARP_OK;
+    auto up = [&](void **dst, const void *src, size_t bytes) {
+        if (st != HARP_OK || !src) return;
+        if (cudaMalloc(dst, std::max<size_t>(bytes, 16)) != cudaSuccess) { st = HARP_ERR_ALLOC; return; }
+        if (cudaMemcpy(*dst, src, bytes, cudaMemcpyHostToDevice) != cudaSuccess) st = HARP_ERR_CUDA;
+    };
+    up(&d_theta, theta ? (const void *)theta : (const void *)theta_q, theta_bytes);
+    if (!theta) up(&d_scales, scales, (size_t)n_blocks * sizeof(float));
+    up(&d_mixer, mixer, (size_t)b * b * sizeof(float));
+    const size_t out_bytes = (size_t)n_blocks * b * b * sizeof(float);
+    if (st == HARP_OK && cudaMalloc(&d_out, std::max<size_t>(out_bytes, 16)) != cudaSuccess) st = HARP_ERR_ALLOC;
+    if (st == HARP_OK)
+        st = harp_blocks_from_theta_device(b, n_blocks, theta ? (const float *)d_theta : nullptr,
+                                           theta ? nullptr : (const int8_t *)d_theta, (const float *)d_scales,
+                                           (const float *)d_mixer, (float *)d_out, nullptr);
+    if (st == HARP_OK && cudaMemcpy(out_host, d_out, out_bytes, cudaMemcpyDeviceToHost) != cudaSuccess) st = HARP_ERR_CUDA;
+    if (st != HARP_OK) cudaGetLastError();
+    cudaFree(d_theta); cudaFree(d_scales); cudaFree(d_mixer); cudaFree(d_out);
+    return st;
+}
+
+}  // namespace
+
 extern "C" harp_status_t harp_plan_create_from_theta(harp_plan_t **out, int64_t d, int32_t n_stages, const int32_t *radices,
                                                      const int32_t *perm, const int8_t *signs, const float *const *theta,
                                                      const int8_t *const *theta_q, const float *const *scales,
@@ -206,9 +243,13 @@ extern "C" harp_status_t harp_plan_create_from_theta(harp_plan_t **out, int64_t 
         } catch (const std::bad_alloc &) {
             return HARP_ERR_ALLOC;
         }
-        const harp_status_t st = harp_blocks_from_theta(b, d / b, theta ? theta[t] : nullptr, theta_q ? theta_q[t] : nullptr,
-                                                        scales ? scales[t] : nullptr, mixers ? mixers[t] : nullptr,
-                                                        blocks[(size_t)t].data());
+        // rebuilt by the device kernels; radices beyond their limit by the host routine
+        harp_status_t st = stage_blocks_on_device(b, d / b, theta ? theta[t] : nullptr, theta_q ? theta_q[t] : nullptr,
+                                                  scales ? scales[t] : nullptr, mixers ? mixers[t] : nullptr,
+                                                  blocks[(size_t)t].data());
+        if (st == HARP_ERR_UNSUPPORTED)
+            st = harp_blocks_from_theta(b, d / b, theta ? theta[t] : nullptr, theta_q ? theta_q[t] : nullptr,
+                                        scales ? scales[t] : nullptr, mixers ? mixers[t] : nullptr, blocks[(size_t)t].data());
         if (st != HARP_OK) return st;
         ptrs[(size_t)t] = blocks[(size_t)t].data();
     }

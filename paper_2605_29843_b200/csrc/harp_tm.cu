@@ -85,9 +85,11 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
 //  the phases), 11 wait for D (phase 2), 12 D -> tile buffer
 __device__ long long g_tm_timing[16];
 #ifdef HARP_TM_TIMING
+#define TM_DECL long long acc[16] = {0}
 #define TM_T(var) const long long var = clock64()
 #define TM_ACC(slot, a, b) acc[slot] += (b) - (a)
 #else
+#define TM_DECL
 #define TM_T(var)
 #define TM_ACC(slot, a, b)
 #endif
@@ -177,7 +179,7 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
         if (lane == 0) {
             int cur_col = -1, slot = 1;
             int64_t issued = 0;
-            long long acc[16] = {0};
+            TM_DECL;
             for (int64_t t = t_begin; t < t_end; ++t) {
                 const int64_t i = t - t_begin;
                 const int b = (int)(i % kNBuf);
@@ -230,7 +232,7 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
             const uint32_t idesc = instr_desc(128, 16);
             int cur_col = -1, slot = 1;
             uint32_t ua = 0;
-            long long acc[16] = {0};
+            TM_DECL;
             for (int64_t t = t_begin; t < t_end; ++t) {
                 const int col = (int)(t / P.n_row_tiles);
                 if (col != cur_col) { cur_col = col; slot ^= 1; }
@@ -267,7 +269,7 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
     } else if (warp == 2) {
         // ---------------- store: finished tiles back to global memory ----------------
         if (lane == 0) {
-            long long acc[16] = {0};
+            TM_DECL;
             for (int64_t t = t_begin; t < t_end; ++t) {
                 const int64_t i = t - t_begin;
                 const int b = (int)(i % kNBuf);
@@ -302,7 +304,7 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
         const int r = ((warp & 3) << 5) | lane;             // row of the tile
         const uint32_t tlane = tmem + ((uint32_t)((warp & 3) << 5) << 16);
         uint32_t ud = 0;
-        long long acc[16] = {0};
+        TM_DECL;
         for (int64_t t = t_begin; t < t_end; ++t) {
             const int64_t i = t - t_begin;
             const int b = (int)(i % kNBuf);
