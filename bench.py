@@ -9,7 +9,10 @@ transpose apply (x = y Q^T) of a batch.  `value` counts row-applies per second
 buffer is touched again only after three others (> 3x the 126 MB L2) have streamed by.
 
 Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead.
-`--all-configs` adds per-configuration measurements under the key "per_config".
+The line carries a compact "per_config" object (forward / transpose rate of all five
+configurations, decode latency, two-sided time; a few repetitions each, full row counts);
+`--all-configs` adds the longer per-configuration measurements (gradient, CUDA-graph decode,
+diagnostics) under "per_config_detail".  `--gpus N` without a launcher starts N ranks itself.
 """
 from __future__ import annotations
 
@@ -33,10 +36,18 @@ METRIC = "harp_apply_rows_per_s"
 UNIT = "rows/s"
 WORKLOAD = "cfg2: d=4096 radix-4 x6, signs + digit-reversal perm, 16384 rows bf16, forward+transpose per step"
 N_BUF = 4
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) per launch of harp_fast_kernel on the
-# headline workload, mean of the forward and the transpose launch in profiles/harp_fast_kernel_cfg2.md
-# (read 134.6 / 134.6 MB, write 75.1 / 75.3 MB: the last tiles' write-back is still in L2 at kernel end).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 209_830_000
+# DRAM bytes per apply (dram__bytes_read.sum + dram__bytes_write.sum, summed over the launches of one
+# apply, mean of forward and transpose) from one ncu capture per configuration of
+# `bench.py --profile-config C --profile-rows R --profile-reps 2`: {config: (R, bytes)}.  Traffic grows in
+# proportion to the rows, so a full launch is scaled by n_rows / R.  Write-back that is still in L2
+# when a kernel ends is not in these figures (cfg1 and cfg2 read below their algorithmic bytes for
+# that reason).
+NCU_TRAFFIC = {1: (4096, 33.8e6), 2: (16384, 209.8e6), 3: (4096, 259.1e6), 4: (4096, 364.2e6), 5: (4096, 833.3e6)}
+
+
+def ncu_traffic(cfg: int, n_rows: int):
+    rows, nbytes = NCU_TRAFFIC[cfg]
+    return nbytes * n_rows / rows
 
 
 def measured_peaks():
@@ -268,11 +279,80 @@ def bench_extra_configs(torch, harp, kernel, peak):
     return out
 
 
+def bench_compact(torch, harp, kernel, peak):
+    """Forward / transpose rate of every configuration at its full row count, decode latency (cfg4,
+    1 and 16 rows) and the two-sided product (cfg5): a few repetitions each, buffers rotated past L2."""
+    out = {}
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(4321)
+    for cfg in (1, 2, 3, 4, 5):
+        w = wl.config(cfg)
+        spec = w.plans["in"] if cfg == 5 else w.plans["q"]
+        data = w.data["x"]
+        plan = harp.plan_from_spec(spec)
+        tdt = torch.float32 if data.dtype == "f32" else torch.bfloat16
+        es = 4 if data.dtype == "f32" else 2
+        nbytes = data.n_rows * data.d * es
+        nbuf = max(2, min(6, int(np.ceil(2.5 * 126e6 / nbytes)) + 1))
+        bufs = [torch.randn((data.n_rows, data.d), generator=gen, device="cuda", dtype=torch.float32).to(tdt)
+                for _ in range(nbuf)]
+        res = {"d": data.d, "n_rows": data.n_rows, "dtype": data.dtype, "algorithmic_bytes": 2 * nbytes,
+               "traffic": ncu_traffic(cfg, data.n_rows)}
+        for name, tr in (("forward", False), ("transpose", True)):
+            for i in range(3):
+                harp.apply_(plan, bufs[i % nbuf], transpose=tr, kernel=kernel)
+            torch.cuda.synchronize()
+            iters = max(4, min(40, int(0.05 / (2 * nbytes / (0.3 * peak * 1e9)))))
+            dt = time_region(torch, lambda i: harp.apply_(plan, bufs[i % nbuf], transpose=tr, kernel=kernel), iters)
+            gbs = 2 * nbytes * iters / dt / 1e9
+            res[name] = {"GBps": round(gbs, 1), "frac": round(gbs / peak, 4), "frac_of_8TBps": round(gbs / 8000.0, 4),
+                         "us": round(1e6 * dt / iters, 2)}
+        if cfg == 4:
+            for n in (1, 16):
+                x = bufs[0][:n]
+                for _ in range(5):
+                    harp.apply_(plan, x, kernel=kernel)
+                torch.cuda.synchronize()
+                dt = time_region(torch, lambda i: harp.apply_(plan, x, kernel=kernel), 100)
+                res[f"decode_{n}_rows_us"] = round(1e6 * dt / 100, 2)
+        if cfg == 5:
+            del bufs
+            torch.cuda.empty_cache()
+            wd = w.data["w"]
+            p_out = harp.plan_from_spec(w.plans["out"])
+            W = (torch.randn((wd.n_rows, wd.d), generator=gen, device="cuda") * 0.02).to(torch.bfloat16)
+            for _ in range(2):
+                harp.two_sided_(W, p_out, plan)
+            torch.cuda.synchronize()
+            l0 = harp.harp_launch_count()
+            dt = time_region(torch, lambda i: harp.two_sided_(W, p_out, plan), 5)
+            wbytes = 2 * wd.n_rows * wd.d * 2
+            res["two_sided"] = {"ms": round(1e3 * dt / 5, 4), "launches": (harp.harp_launch_count() - l0) // 5,
+                                "algorithmic_bytes": wbytes, "frac_vs_1R1W": round(wbytes * 5 / dt / 1e9 / peak, 4)}
+        out[f"cfg{cfg}"] = res
+        bufs = None
+        torch.cuda.empty_cache()
+    return out
+
+
+def relaunch_with_ranks(args):
+    """`--gpus N` (N > 1) outside a launcher: start N ranks of this script on this node."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd))
+
+
 def run_gpu(args):
     import torch
     import torch.distributed as dist
     import paper_2605_29843_b200 as harp
 
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        relaunch_with_ranks(args)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -282,8 +362,7 @@ def run_gpu(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     harp.lib()
-    kernel = {"auto": harp.KERNEL_AUTO, "generic": harp.KERNEL_GENERIC, "fast": harp.KERNEL_FAST,
-              "split": harp.KERNEL_SPLIT}[args.kernel]
+    kernel = KERNELS(harp)[args.kernel]
 
     w = wl.config(2)
     spec, data = w.plans["q"], w.data["x"]
@@ -353,7 +432,8 @@ def run_gpu(args):
             "ms_per_step": 1e3 * dt_max / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "n_rows": n_rows, "d": d, "kernel": args.kernel,
-                       "arithmetic": "bf16 operands, fp32 accumulate, one rounding to bf16 per phase",
+                       "arithmetic": "bf16 operands (fused blocks rounded to bf16 at plan time), fp32 accumulate, "
+                                     "rows rounded to bf16 after each of the three fused phases",
                        "l2": f"{N_BUF} rotating 134 MB buffers (inputs larger than L2)", "parallelism": f"rows x{world}"},
             "clocks": clocks,
             "e2e": {"value": world * 2 * n_rows * e2e_steps / e2e_dt, "unit": UNIT,
@@ -362,19 +442,27 @@ def run_gpu(args):
             "gpu_launches": int(launches),
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                          "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBps": achieved / 8000.0,
-                         "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                         "traffic": ncu_traffic(2, n_rows),
                          "algorithmic_bytes_per_launch": n_rows * row_bytes,
                          "us_per_launch": 1e6 * per_launch_s},
         }
         if not args.no_cpu and world == 1:
             line["cpu_baseline"] = cpu_baseline(spec, data)
-        if args.all_configs and world == 1:
-            del bufs
+        if world == 1 and not args.no_per_config:
+            del bufs, pinned
             torch.cuda.empty_cache()
-            line["per_config"] = bench_extra_configs(torch, harp, kernel, peak)
+            line["per_config"] = bench_compact(torch, harp, kernel, peak)
+        if args.all_configs and world == 1:
+            torch.cuda.empty_cache()
+            line["per_config_detail"] = bench_extra_configs(torch, harp, kernel, peak)
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+def KERNELS(harp):
+    return {"auto": harp.KERNEL_AUTO, "generic": harp.KERNEL_GENERIC, "fast": harp.KERNEL_FAST,
+            "split": harp.KERNEL_SPLIT, "tmem": harp.KERNEL_TMEM}
 
 
 def run_profile_case(args):
@@ -382,8 +470,7 @@ def run_profile_case(args):
     `--profile-rows` seeded device rows, alternating forward and transpose, `--profile-reps` times."""
     import torch
     import paper_2605_29843_b200 as harp
-    kernel = {"auto": harp.KERNEL_AUTO, "generic": harp.KERNEL_GENERIC, "fast": harp.KERNEL_FAST,
-              "split": harp.KERNEL_SPLIT}[args.kernel]
+    kernel = KERNELS(harp)[args.kernel]
     gen = torch.Generator(device="cuda")
     gen.manual_seed(7)
     if args.profile_config == 6:          # two-sided processing of configuration 5's weight matrix
@@ -425,7 +512,8 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="harp", choices=["harp", "reference"])
-    ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "fast", "split"])
+    ap.add_argument("--kernel", default="auto", choices=["auto", "generic", "fast", "split", "tmem"])
+    ap.add_argument("--no-per-config", action="store_true", help="headline only: skip the compact per-configuration block")
     ap.add_argument("--profile-config", type=int, default=0, help="run a small profiling case of this configuration and exit")
     ap.add_argument("--profile-rows", type=int, default=8192)
     ap.add_argument("--profile-reps", type=int, default=2)
