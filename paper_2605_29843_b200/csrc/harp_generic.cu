@@ -309,9 +309,10 @@ __device__ __forceinline__ float4 f4_fma(float4 a, float k, float4 c) {
 }
 
 template <int B>
-__device__ __forceinline__ void stage_blocks_t(float *v, int n_rg, int R4, int d, int s, const float *__restrict__ Kt, int transpose) {
+__device__ __forceinline__ void stage_blocks_t(float *v, int n_rg, int R4, int d, int s, const float *__restrict__ Kt, int transpose,
+                                               int tid, int nthr) {
     const int nblk = d / B;
-    for (int c = threadIdx.x; c < nblk; c += blockDim.x) {
+    for (int c = tid; c < nblk; c += nthr) {
         const int alpha = c / s, beta = c - alpha * s;
         const int base = alpha * B * s + beta;
         int pos[B];
@@ -339,21 +340,193 @@ __device__ __forceinline__ void stage_blocks_t(float *v, int n_rg, int R4, int d
     }
 }
 
-template <typename T, int NT, bool BIG>
-__global__ void __launch_bounds__(NT, 1)
+
+// ---- the two ends of the stage list done on the way in / out of the transposed tile ----------------
+// Stage 0 of the table (stride 1, radix 4): a thread that copies the quad of coordinates 4m .. 4m+3 of
+// four rows between global memory and the tile owns block m of that stage, so the stage is applied in
+// registers during the copy: forward on the way in (after the signs), transpose on the way out (before
+// them).  One shared-memory pass and one barrier less, and the arithmetic runs under the HBM transfer.
+template <typename T>
+__device__ __forceinline__ void copy_in_with_stage0(const T *xt, float *v, int rows, int n_rg, int R4, int d,
+                                                    const float *__restrict__ Kt, const int8_t *__restrict__ signs, int tid, int nthr) {
+    const int nq = d >> 2;
+    for (int m = tid; m < nq; m += nthr) {
+        float K[4][4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float sg = (signs && signs[4 * m + i] < 0) ? -1.f : 1.f;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) K[i][j] = sg * __ldg(Kt + (size_t)(i * 4 + j) * nq + m);     // sign folded into the row
+        }
+        int pos[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) pos[j] = tpos(4 * m + j) * R4;
+        float e[4][4], nx[4][4];
+#pragma unroll
+        for (int rr = 0; rr < 4; ++rr) {
+            if (rr < rows) load4<T>(xt + (int64_t)rr * d + 4 * m, e[rr]);
+            else e[rr][0] = e[rr][1] = e[rr][2] = e[rr][3] = 0.f;
+        }
+        for (int rg = 0; rg < n_rg; ++rg) {
+            if (rg + 1 < n_rg) {                        // next row group in flight while this one is multiplied
+#pragma unroll
+                for (int rr = 0; rr < 4; ++rr) {
+                    if (4 * (rg + 1) + rr < rows) load4<T>(xt + (int64_t)(4 * (rg + 1) + rr) * d + 4 * m, nx[rr]);
+                    else nx[rr][0] = nx[rr][1] = nx[rr][2] = nx[rr][3] = 0.f;
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float4 a = f4_scale(make_float4(e[0][0], e[1][0], e[2][0], e[3][0]), K[0][j]);
+#pragma unroll
+                for (int i = 1; i < 4; ++i) a = f4_fma(make_float4(e[0][i], e[1][i], e[2][i], e[3][i]), K[i][j], a);
+                *reinterpret_cast<float4 *>(v + pos[j] + 4 * rg) = a;
+            }
+#pragma unroll
+            for (int rr = 0; rr < 4; ++rr)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) e[rr][i] = nx[rr][i];
+        }
+    }
+}
+
+template <typename T>
+__device__ __forceinline__ void copy_out_with_stage0(T *xt, const float *v, int rows, int n_rg, int R4, int d,
+                                                     const float *__restrict__ Kt, const int8_t *__restrict__ signs, int tid, int nthr) {
+    const int nq = d >> 2;
+    for (int m = tid; m < nq; m += nthr) {
+        float K[4][4];                                  // K[i][j] of the transposed block, sign of output j folded in
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const float sg = (signs && signs[4 * m + j] < 0) ? -1.f : 1.f;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) K[i][j] = sg * __ldg(Kt + (size_t)(j * 4 + i) * nq + m);
+        }
+        int pos[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) pos[j] = tpos(4 * m + j) * R4;
+        for (int rg = 0; rg < n_rg; ++rg) {
+            float4 in[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) in[i] = *reinterpret_cast<const float4 *>(v + pos[i] + 4 * rg);
+            float4 o[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                float4 a = f4_scale(in[0], K[0][j]);
+#pragma unroll
+                for (int i = 1; i < 4; ++i) a = f4_fma(in[i], K[i][j], a);
+                o[j] = a;
+            }
+            const float e[4][4] = {{o[0].x, o[1].x, o[2].x, o[3].x}, {o[0].y, o[1].y, o[2].y, o[3].y},
+                                   {o[0].z, o[1].z, o[2].z, o[3].z}, {o[0].w, o[1].w, o[2].w, o[3].w}};
+#pragma unroll
+            for (int rr = 0; rr < 4; ++rr)
+                if (4 * rg + rr < rows) store4<T>(xt + (int64_t)(4 * rg + rr) * d + 4 * m, e[rr]);
+        }
+    }
+}
+
+// The top stage of the table (stride >= 32, so neighbouring lanes own neighbouring coordinates): its
+// results go from registers straight to global memory (forward), or its operands come straight from
+// global memory (transpose); a warp moves 128 contiguous bytes of a row per access.
+template <typename T, int B>
+__device__ __forceinline__ void stage_to_global(T *xt, const float *v, int rows, int n_rg, int R4, int d, int s,
+                                                const float *__restrict__ Kt, int tid, int nthr) {
+    const int nblk = d / B;
+    for (int c = tid; c < nblk; c += nthr) {
+        const int alpha = c / s, beta = c - alpha * s;
+        const int base = alpha * B * s + beta;
+        int pos[B];
+#pragma unroll
+        for (int i = 0; i < B; ++i) pos[i] = tpos(base + i * s) * R4;
+        float K[B][B];
+#pragma unroll
+        for (int i = 0; i < B; ++i)
+#pragma unroll
+            for (int j = 0; j < B; ++j) K[i][j] = __ldg(Kt + (size_t)(i * B + j) * nblk + c);
+        for (int rg = 0; rg < n_rg; ++rg) {
+            float4 in[B];
+#pragma unroll
+            for (int i = 0; i < B; ++i) in[i] = *reinterpret_cast<const float4 *>(v + pos[i] + 4 * rg);
+#pragma unroll
+            for (int j = 0; j < B; ++j) {
+                float4 a = f4_scale(in[0], K[0][j]);
+#pragma unroll
+                for (int i = 1; i < B; ++i) a = f4_fma(in[i], K[i][j], a);
+                T *dst = xt + (int64_t)(4 * rg) * d + base + j * s;
+                const float o[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+                for (int rr = 0; rr < 4; ++rr)
+                    if (4 * rg + rr < rows) dst[(int64_t)rr * d] = from_f32<T>(o[rr]);
+            }
+        }
+    }
+}
+
+template <typename T, int B>
+__device__ __forceinline__ void stage_from_global(const T *xt, float *v, int rows, int n_rg, int R4, int d, int s,
+                                                  const float *__restrict__ Kt, int tid, int nthr) {
+    const int nblk = d / B;
+    for (int c = tid; c < nblk; c += nthr) {
+        const int alpha = c / s, beta = c - alpha * s;
+        const int base = alpha * B * s + beta;
+        int pos[B];
+#pragma unroll
+        for (int i = 0; i < B; ++i) pos[i] = tpos(base + i * s) * R4;
+        float K[B][B];                                  // transposed block
+#pragma unroll
+        for (int i = 0; i < B; ++i)
+#pragma unroll
+            for (int j = 0; j < B; ++j) K[i][j] = __ldg(Kt + (size_t)(j * B + i) * nblk + c);
+#pragma unroll 2
+        for (int rg = 0; rg < n_rg; ++rg) {
+            float4 in[B];
+#pragma unroll
+            for (int i = 0; i < B; ++i) {
+                const T *src = xt + (int64_t)(4 * rg) * d + base + i * s;
+                float e[4];
+#pragma unroll
+                for (int rr = 0; rr < 4; ++rr) e[rr] = 4 * rg + rr < rows ? to_f32<T>(src[(int64_t)rr * d]) : 0.f;
+                in[i] = make_float4(e[0], e[1], e[2], e[3]);
+            }
+#pragma unroll
+            for (int j = 0; j < B; ++j) {
+                float4 a = f4_scale(in[0], K[0][j]);
+#pragma unroll
+                for (int i = 1; i < B; ++i) a = f4_fma(in[i], K[i][j], a);
+                *reinterpret_cast<float4 *>(v + pos[j] + 4 * rg) = a;
+            }
+        }
+    }
+}
+
+template <typename T, int NT, bool BIG, int MINB>
+__global__ void __launch_bounds__(NT, MINB)
 harp_rowvec_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_cta, int R4, StageTable st,
                    const float *__restrict__ blocks, const int32_t *__restrict__ perm,
-                   const int8_t *__restrict__ signs, int transpose) {
+                   const int8_t *__restrict__ signs, int transpose, int fuse_lo, int fuse_hi) {
     extern __shared__ __align__(16) float v[];       // [d][R4]
     const int64_t row0 = (int64_t)blockIdx.x * rows_per_cta;
     const int rows = (int)min((int64_t)rows_per_cta, n_rows - row0);
     const int n_rg = (rows + 3) >> 2;
     T *xt = x + row0 * d;
+    const int tid = threadIdx.x, nthr = NT;
     const bool aligned = d % 4 == 0 && (reinterpret_cast<uintptr_t>(x) % (4 * sizeof(T))) == 0;
+    // fuse_lo / fuse_hi (host: no permutation, aligned rows): stage 0 and the top stage run on the way
+    // in and out of the tile
+    const int top = st.m - 1;
     // a1-a3: load, sign, gather (forward) -- or plain load (transpose)
-    if (aligned && (transpose || !perm)) {
+    if (!transpose && fuse_lo) {
+        copy_in_with_stage0<T>(xt, v, rows, n_rg, R4, d, blocks + st.off[0], signs, tid, nthr);
+    } else if (transpose && fuse_hi) {
+        const float *Kt = blocks + st.off[top];
+        const int b = st.b[top];
+        if (b == 2) stage_from_global<T, 2>(xt, v, rows, n_rg, R4, d, st.s[top], Kt, tid, nthr);
+        else if (b == 3) stage_from_global<T, 3>(xt, v, rows, n_rg, R4, d, st.s[top], Kt, tid, nthr);
+        else stage_from_global<T, 4>(xt, v, rows, n_rg, R4, d, st.s[top], Kt, tid, nthr);
+    } else if (aligned && (transpose || !perm)) {
         const int nq = d >> 2;
-        for (int w = threadIdx.x; w < nq * n_rg; w += NT) {
+        for (int w = tid; w < nq * n_rg; w += nthr) {
             const int rg = w / nq, m = w - rg * nq;
             float e[4][4];
 #pragma unroll
@@ -369,7 +542,7 @@ harp_rowvec_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_cta, i
             }
         }
     } else {
-        for (int w = threadIdx.x; w < d * n_rg; w += NT) {
+        for (int w = tid; w < d * n_rg; w += nthr) {
             const int rg = w / d, i = w - rg * d;
             const int src = (!transpose && perm) ? perm[i] : i;
             const float sg = (!transpose && signs && signs[src] < 0) ? -1.f : 1.f;
@@ -382,23 +555,32 @@ harp_rowvec_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_cta, i
     __syncthreads();
     for (int k = 0; k < st.m; ++k) {
         const int t = transpose ? st.m - 1 - k : k;
+        if ((t == 0 && fuse_lo) || (t == top && fuse_hi)) continue;      // done during a copy
         const float *Kt = blocks + st.off[t];
         const int b = st.b[t];
-        if (b == 2) stage_blocks_t<2>(v, n_rg, R4, d, st.s[t], Kt, transpose);
-        else if (b == 3) stage_blocks_t<3>(v, n_rg, R4, d, st.s[t], Kt, transpose);
-        else if (b == 4) stage_blocks_t<4>(v, n_rg, R4, d, st.s[t], Kt, transpose);
+        if (b == 2) stage_blocks_t<2>(v, n_rg, R4, d, st.s[t], Kt, transpose, tid, nthr);
+        else if (b == 3) stage_blocks_t<3>(v, n_rg, R4, d, st.s[t], Kt, transpose, tid, nthr);
+        else if (b == 4) stage_blocks_t<4>(v, n_rg, R4, d, st.s[t], Kt, transpose, tid, nthr);
         else if (BIG) {
-            if (b == 5) stage_blocks_t<5>(v, n_rg, R4, d, st.s[t], Kt, transpose);
-            else if (b == 6) stage_blocks_t<6>(v, n_rg, R4, d, st.s[t], Kt, transpose);
-            else if (b == 7) stage_blocks_t<7>(v, n_rg, R4, d, st.s[t], Kt, transpose);
-            else stage_blocks_t<8>(v, n_rg, R4, d, st.s[t], Kt, transpose);
+            if (b == 5) stage_blocks_t<5>(v, n_rg, R4, d, st.s[t], Kt, transpose, tid, nthr);
+            else if (b == 6) stage_blocks_t<6>(v, n_rg, R4, d, st.s[t], Kt, transpose, tid, nthr);
+            else if (b == 7) stage_blocks_t<7>(v, n_rg, R4, d, st.s[t], Kt, transpose, tid, nthr);
+            else stage_blocks_t<8>(v, n_rg, R4, d, st.s[t], Kt, transpose, tid, nthr);
         }
         __syncthreads();
     }
     // a5: store -- or scatter and sign (transpose)
-    if (aligned && (!transpose || !perm)) {
+    if (transpose && fuse_lo) {
+        copy_out_with_stage0<T>(xt, v, rows, n_rg, R4, d, blocks + st.off[0], signs, tid, nthr);
+    } else if (!transpose && fuse_hi) {
+        const float *Kt = blocks + st.off[top];
+        const int b = st.b[top];
+        if (b == 2) stage_to_global<T, 2>(xt, v, rows, n_rg, R4, d, st.s[top], Kt, tid, nthr);
+        else if (b == 3) stage_to_global<T, 3>(xt, v, rows, n_rg, R4, d, st.s[top], Kt, tid, nthr);
+        else stage_to_global<T, 4>(xt, v, rows, n_rg, R4, d, st.s[top], Kt, tid, nthr);
+    } else if (aligned && (!transpose || !perm)) {
         const int nq = d >> 2;
-        for (int w = threadIdx.x; w < nq * n_rg; w += NT) {
+        for (int w = tid; w < nq * n_rg; w += nthr) {
             const int rg = w / nq, m = w - rg * nq;
             float4 q[4];
 #pragma unroll
@@ -413,7 +595,7 @@ harp_rowvec_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_cta, i
                 if (4 * rg + rr < rows) store4<T>(xt + (int64_t)(4 * rg + rr) * d + 4 * m, e[rr]);
         }
     } else {
-        for (int w = threadIdx.x; w < d * n_rg; w += NT) {
+        for (int w = tid; w < d * n_rg; w += nthr) {
             const int rg = w / d, i = w - rg * d;
             const int dst = (transpose && perm) ? perm[i] : i;
             const float sg = (transpose && signs && signs[dst] < 0) ? -1.f : 1.f;
@@ -426,10 +608,10 @@ harp_rowvec_kernel(T *__restrict__ x, int64_t n_rows, int d, int rows_per_cta, i
     }
 }
 
-template <typename T, int NT, bool BIG>
+template <typename T, int NT, bool BIG, int MINB = 1>
 harp_status_t launch_rowvec(const harp_plan *plan, const StageTable &st, const float *blocks, void *x, int64_t n_rows,
                             int transpose, cudaStream_t stream) {
-    auto kern = harp_rowvec_kernel<T, NT, BIG>;
+    auto kern = harp_rowvec_kernel<T, NT, BIG, MINB>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
         return HARP_ERR_CUDA;
     int dev = 0, sms = 148;
@@ -438,17 +620,24 @@ harp_status_t launch_rowvec(const harp_plan *plan, const StageTable &st, const f
     const int64_t d = plan->d;
     // groups of four rows per CTA: an odd number (bank spread), as many as shared memory holds,
     // but no more than one wave of CTAs needs
-    int64_t g_max = (226 * 1024) / (d * 16);
+    // MINB CTAs share an SM (and its shared memory): while one multiplies, another copies
+    int64_t g_max = (226 * 1024 / MINB) / (d * 16);
     if (g_max % 2 == 0) --g_max;
     if (g_max < 1) return HARP_ERR_UNSUPPORTED;
-    int64_t g = ((n_rows + sms - 1) / sms + 3) / 4;
+    int64_t g = ((n_rows + (int64_t)sms * MINB - 1) / ((int64_t)sms * MINB) + 3) / 4;
     g = std::max<int64_t>(1, std::min<int64_t>(g, std::min<int64_t>(g_max, 15)));
     const int64_t g_pad = g | 1;                     // g_pad <= g_max because g_max is odd
     const int64_t r = 4 * g;
     const int64_t grid = (n_rows + r - 1) / r;
     if (grid > 0x7fffffffLL) return HARP_ERR_BAD_DIM;
+    // the ends of the stage list on the way in and out: identity permutation, aligned rows, stage 0 of
+    // radix 4 and stride 1, a top stage of radix <= 4 whose stride keeps a warp's accesses contiguous,
+    // at least three stages (so that the two ends are different stages with a barrier between them)
+    const bool ends_ok = !plan->d_perm && d % 4 == 0 && (reinterpret_cast<uintptr_t>(x) % (4 * sizeof(T))) == 0 && st.m >= 3;
+    const int fuse_lo = ends_ok && st.b[0] == 4 && st.s[0] == 1;
+    const int fuse_hi = ends_ok && st.b[st.m - 1] <= 4 && st.s[st.m - 1] >= 32;
     kern<<<(unsigned)grid, NT, (size_t)d * 16 * g_pad, stream>>>((T *)x, n_rows, (int)d, (int)r, (int)(4 * g_pad), st, blocks,
-                                                              plan->d_perm, plan->d_signs, transpose);
+                                                              plan->d_perm, plan->d_signs, transpose, fuse_lo, fuse_hi);
     g_harp_launches.fetch_add(1, std::memory_order_relaxed);
     return cudaGetLastError() == cudaSuccess ? HARP_OK : HARP_ERR_CUDA;
 }
