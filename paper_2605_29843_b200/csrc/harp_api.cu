@@ -210,7 +210,14 @@ extern "C" harp_status_t harp_apply_ex(const harp_plan_t *plan, void *x, int64_t
     if (kernel == HARP_KERNEL_FAST) return harp_fast_apply(plan, x, n_rows, dtype, transpose, s);
     if (kernel == HARP_KERNEL_SPLIT) return harp_split_apply(plan, x, n_rows, dtype, transpose, s);
     if (kernel == HARP_KERNEL_TMEM) return harp_tm_apply(plan, x, n_rows, dtype, transpose, s);
-    harp_status_t st = harp_fast_apply(plan, x, n_rows, dtype, transpose, s);
+    harp_status_t st;
+    if (plan->d == 256 && n_rows >= 1024) {
+        // one pass of the tensor-memory kernel covers the whole processor: several times the rate of the
+        // 16-row tile kernels, whose per-tile block-kernel traffic dominates at this width
+        st = harp_tm_apply(plan, x, n_rows, dtype, transpose, s);
+        if (st != HARP_ERR_UNSUPPORTED) return st;
+    }
+    st = harp_fast_apply(plan, x, n_rows, dtype, transpose, s);
     if (st != HARP_ERR_UNSUPPORTED) return st;
     st = harp_split_apply(plan, x, n_rows, dtype, transpose, s);
     if (st != HARP_ERR_UNSUPPORTED) return st;

@@ -86,6 +86,10 @@ void harp_tm_destroy(harp_plan *plan);
 harp_status_t harp_tm_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype,
                             int transpose, cudaStream_t stream);
 int32_t harp_tm_error_word(const harp_plan *plan);
+// the stages below stride 256 alone (lower pass of the two-pass paths); 0 stages = not available
+int harp_tm_slab_stages(const harp_plan *plan);
+harp_status_t harp_tm_slab_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype,
+                                 int transpose, cudaStream_t stream);
 
 // column-side apply for two-sided processing (harp_col.cu): plan applied down the columns of a
 // dim(plan) x n_cols row-major matrix with leading dimension ld

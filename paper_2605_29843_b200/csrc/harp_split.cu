@@ -433,6 +433,7 @@ struct SplitPlan {
     std::vector<void *> dev_allocs;
     int64_t chunk_rows = 0;    // rows per L2-resident chunk
     int sms = 148;
+    int lower_stages = 0;      // pass[0] covers stages [0, lower_stages)
     // dense upper pass (replaces pass[1] when set)
     bool dense_upper = false;
     UpperPass up_fwd{}, up_bwd{};
@@ -746,6 +747,7 @@ harp_status_t harp_split_build(harp_plan *plan) {
 
     SplitPlan *sp = new (std::nothrow) SplitPlan();
     if (!sp) return HARP_ERR_ALLOC;
+    sp->lower_stages = lower.back().t1;
     harp_status_t st = build_pass(plan, sp, sp->pass[0], lower, true, S_mid, U, 1);
     if (st == HARP_OK && want_dense) st = build_dense_upper(plan, sp, lower.back().t1, S_mid, U);
     else if (st == HARP_OK && !upper.empty()) st = build_pass(plan, sp, sp->pass[1], upper, false, S_mid, U, Lw);
@@ -808,6 +810,7 @@ cudaError_t launch_pass(void (*kern)(__nv_bfloat16 *, int64_t, int64_t, PassT), 
 }
 
 constexpr int64_t kOverlapMaxRows = 64;
+constexpr int64_t kTmSlabMinRows = 1024;
 
 harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype, int transpose,
                                cudaStream_t stream) {
@@ -839,6 +842,13 @@ harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, h
                 g_harp_launches.fetch_add(1, std::memory_order_relaxed);
                 if (err != cudaSuccess || cudaGetLastError() != cudaSuccess) return HARP_ERR_CUDA;
                 continue;
+            }
+            // lower pass on slabs of 256 coordinates: the tensor-memory kernel (128-row tiles, bulk tensor
+            // copies) when the plan has it and the batch fills its tiles
+            if (pi == 0 && r1 - r0 >= kTmSlabMinRows && harp_tm_slab_stages(plan) == sp->lower_stages) {
+                const harp_status_t ts = harp_tm_slab_apply(plan, xb + r0 * plan->d, r1 - r0, dtype, transpose, stream);
+                if (ts == HARP_OK) continue;
+                if (ts != HARP_ERR_UNSUPPORTED) return ts;
             }
             const PassHost &ph = sp->pass[pi];
             const SplitPass &P = transpose ? ph.bwd : ph.fwd;

@@ -430,7 +430,13 @@ struct TmPass {
 }  // namespace
 
 struct TmPlan {
-    std::vector<TmPass> pass[2];     // [0] forward, [1] transpose
+    std::vector<TmPass> pass[2];     // [0] forward, [1] transpose: the whole processor (empty if only the slab part exists)
+    // the stages below stride 256 alone, on slabs of 256 contiguous coordinates (any d that is a multiple
+    // of 256, identity permutation): the first pass of the two-pass paths for wide rows
+    TmPass slab[2];
+    bool has_slab = false;
+    bool slab_shared = false;        // slab[] are copies of entries of pass[] (natural order, d = 256 or 4096)
+    int slab_stages = 0;             // stages [0, slab_stages) are the slab's
     int32_t *d_err = nullptr;
     int n_sm = 0;
 };
@@ -469,16 +475,17 @@ struct Builder {
     Held held[3];                     // state of the memory positions
     int final_tab[3][16];             // transpose direction: table each digit must end with
     int dir;                          // 0 forward, 1 transpose
+    int64_t wide_cols = 0;            // > 0: a slab pass of a wide row, tile column c = coordinates [256 c, 256 c + 256)
     std::vector<uint8_t> img;
 
     int64_t perm_of(int64_t i) const { return plan->h_perm.empty() ? i : plan->h_perm[(size_t)i]; }
     double sign_of(int64_t i) const { return plan->h_signs.empty() ? 1.0 : (double)plan->h_signs[(size_t)perm_of(i)]; }
 
     // fragments of one pass; positions: inner = 0, outer = po, tile column = the remaining position(s)
-    bool add_pass(TmPlan *tp, int fmt, int k0, int k1, int xpose) {
+    bool add_pass(TmPlan *tp, int fmt, int k0, int k1, int xpose, TmPass *slab_out = nullptr) {
         const int po = fmt == FMT_C ? 1 : 2;                 // outer position
         const int pc = n_dig == 2 ? -1 : (fmt == FMT_C ? 2 : 1);   // position indexing the tile column
-        const int n_col = pc < 0 ? 1 : 16;
+        const int n_col = wide_cols > 0 ? (int)wide_cols : (pc < 0 ? 1 : 16);
         const int nph = k1 < 0 ? 1 : 2;
         img.assign((size_t)n_col * nph * kFragBytes, 0);
         Held h[3] = {held[0], held[1], held[2]};
@@ -494,7 +501,8 @@ struct Builder {
             for (int col = 0; col < n_col; ++col)
                 for (int blk = 0; blk < 16; ++blk) {
                     int64_t base = (int64_t)h[pb].tab[blk] * (phase[h[pb].digit].S);
-                    if (pc >= 0) base += (int64_t)h[pc].tab[col] * (phase[h[pc].digit].S);
+                    if (wide_cols > 0) base += (int64_t)col * 256;
+                    else if (pc >= 0) base += (int64_t)h[pc].tab[col] * (phase[h[pc].digit].S);
                     harp_fuse::fused_block(plan, hp, base, F);          // F[in][out] of the forward map
                     uint8_t *dst = img.data() + ((size_t)col * nph + ph) * kFragBytes + (size_t)blk * 512;
                     for (int n = 0; n < 16; ++n)
@@ -520,7 +528,8 @@ struct Builder {
         ps.fmt = fmt; ps.k0 = k0; ps.k1 = k1; ps.xpose = xpose;
         ps.n_col_tiles = n_col; ps.lo_count = 16;
         if (cudaMalloc(&ps.d_frags, img.size()) != cudaSuccess) { cudaGetLastError(); return false; }
-        tp->pass[dir].push_back(ps);
+        if (slab_out) *slab_out = ps;
+        else tp->pass[dir].push_back(ps);
         if (cudaMemcpy(ps.d_frags, img.data(), img.size(), cudaMemcpyHostToDevice) != cudaSuccess) return false;
         return true;
     }
@@ -545,6 +554,8 @@ void harp_tm_destroy(harp_plan *plan) {
     for (int dir = 0; dir < 2; ++dir)
         for (TmPass &p : plan->tm->pass[dir])
             if (p.d_frags) cudaFree(p.d_frags);
+    for (int dir = 0; dir < 2; ++dir)
+        if (!plan->tm->slab_shared && plan->tm->slab[dir].d_frags) cudaFree(plan->tm->slab[dir].d_frags);
     if (plan->tm->d_err) cudaFree(plan->tm->d_err);
     delete plan->tm;
     plan->tm = nullptr;
@@ -552,21 +563,51 @@ void harp_tm_destroy(harp_plan *plan) {
 
 harp_status_t harp_tm_build(harp_plan *plan) {
     const int64_t d = plan->d;
-    if (d != 256 && d != 4096) return HARP_ERR_UNSUPPORTED;
+    if (d % 256 != 0) return HARP_ERR_UNSUPPORTED;
     if (!encode_fn()) return HARP_ERR_UNSUPPORTED;
+    const bool whole = d == 256 || d == 4096;        // the whole processor as passes of this path
     const int n_dig = d == 256 ? 2 : 3;
-    // group the stages into phases whose radices multiply to 16
+    // group the stages into phases whose radices multiply to 16 (all of them, or the two below stride 256)
     Builder bld;
     bld.plan = plan;
-    bld.n_dig = n_dig;
+    bld.n_dig = whole ? n_dig : 2;
     int t = 0;
-    for (int dg = 0; dg < n_dig; ++dg) {
+    for (int dg = 0; dg < (whole ? n_dig : 2); ++dg) {
         int prod = 1, t0 = t;
         while (t < plan->st.m && prod < 16) prod *= plan->st.b[t++];
         if (prod != 16) return HARP_ERR_UNSUPPORTED;
         bld.phase[dg] = harp_fuse::HostPhase{t0, t, 16, plan->st.s[t0], 0, 1};
     }
-    if (t != plan->st.m) return HARP_ERR_UNSUPPORTED;
+    if (whole && t != plan->st.m) return HARP_ERR_UNSUPPORTED;
+    if (!whole) {
+        // wide row: only the slab part, identity permutation
+        if (!plan->h_perm.empty()) return HARP_ERR_UNSUPPORTED;
+        TmPlan *tp = new (std::nothrow) TmPlan();
+        if (!tp) return HARP_ERR_ALLOC;
+        plan->tm = tp;
+        Held ident[3];
+        for (int p = 0; p < 3; ++p) { ident[p].digit = p; for (int v = 0; v < 16; ++v) ident[p].tab[v] = v; }
+        for (int dg = 0; dg < 2; ++dg)
+            for (int v = 0; v < 16; ++v) bld.final_tab[dg][v] = v;
+        bld.wide_cols = d / 256;
+        bool ok = true;
+        for (int dir = 0; dir < 2 && ok; ++dir) {
+            bld.dir = dir;
+            for (int p = 0; p < 3; ++p) bld.held[p] = ident[p];
+            ok = dir == 0 ? bld.add_pass(tp, FMT_C, TM_I, TM_O, 0, &tp->slab[0]) : bld.add_pass(tp, FMT_C, TM_O, TM_I, 0, &tp->slab[1]);
+        }
+        tp->has_slab = ok;
+        tp->slab_stages = t;
+        if (ok && cudaMalloc(&tp->d_err, sizeof(int32_t)) != cudaSuccess) ok = false;
+        if (ok && cudaMemset(tp->d_err, 0, sizeof(int32_t)) != cudaSuccess) ok = false;
+        if (ok && cudaDeviceGetAttribute(&tp->n_sm, cudaDevAttrMultiProcessorCount, plan->device) != cudaSuccess) ok = false;
+        if (!ok) {
+            cudaGetLastError();
+            harp_tm_destroy(plan);
+            return HARP_ERR_ALLOC;
+        }
+        return HARP_OK;
+    }
     // the permutation must move whole 16-ary digits: position digit p of perm[i] depends on one digit of i
     Held init[3];
     int pos_of_digit[3] = {-1, -1, -1};
@@ -629,6 +670,13 @@ harp_status_t harp_tm_build(harp_plan *plan) {
         ok = ok && bld.add_pass(tp, FMT_C, TM_O, -1, 0);
         ok = ok && bld.add_pass(tp, FMT_S, TM_I, -1, 1);
     }
+    if (ok && natural && plan->h_perm.empty()) {
+        // the pass over contiguous slabs is also the lower pass of the two-pass path
+        tp->slab[0] = tp->pass[0].front();
+        tp->slab[1] = tp->pass[1].back();
+        tp->has_slab = tp->slab_shared = true;
+        tp->slab_stages = bld.phase[1].t1;
+    }
     if (ok && cudaMalloc(&tp->d_err, sizeof(int32_t)) != cudaSuccess) ok = false;
     if (ok && cudaMemset(tp->d_err, 0, sizeof(int32_t)) != cudaSuccess) ok = false;
     if (ok && cudaDeviceGetAttribute(&tp->n_sm, cudaDevAttrMultiProcessorCount, plan->device) != cudaSuccess) ok = false;
@@ -640,59 +688,92 @@ harp_status_t harp_tm_build(harp_plan *plan) {
     return HARP_OK;
 }
 
-harp_status_t harp_tm_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype, int transpose,
-                            cudaStream_t stream) {
-    const TmPlan *tp = plan->tm;
-    if (!tp || dtype != HARP_BF16) return HARP_ERR_UNSUPPORTED;
-    if ((reinterpret_cast<uintptr_t>(x) & 15u) != 0) return HARP_ERR_UNSUPPORTED;
-    if (n_rows > (int64_t)1 << 30) return HARP_ERR_UNSUPPORTED;
+namespace {
+
+// tensor maps of one call: rows as 2-D boxes of 64 columns, and (d > 256) as 16 runs of 16 per row
+harp_status_t encode_maps(void *x, int64_t n_rows, int64_t d, bool need_s, CUtensorMap *map_c, CUtensorMap *map_s) {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return HARP_ERR_UNSUPPORTED;
-    const int64_t d = plan->d;
     const cuuint32_t ones[3] = {1, 1, 1};
-    CUtensorMap map_c, map_s;
     {
         const cuuint64_t gdim[2] = {(cuuint64_t)d, (cuuint64_t)n_rows};
         const cuuint64_t gstr[1] = {(cuuint64_t)d * 2};
         const cuuint32_t box[2] = {64, 128};
-        if (enc(&map_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, x, gdim, gstr, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        if (enc(map_c, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, x, gdim, gstr, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return HARP_ERR_CUDA;
     }
-    if (d > 256) {
+    if (need_s) {
         // coordinates as (e within a run of 256, row, run): 16 elements of each of 16 runs per row
         const cuuint64_t gdim[3] = {256, (cuuint64_t)n_rows, (cuuint64_t)(d / 256)};
         const cuuint64_t gstr[2] = {(cuuint64_t)d * 2, 512};
         const cuuint32_t box[3] = {16, 128, 16};
-        if (enc(&map_s, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, x, gdim, gstr, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
+        if (enc(map_s, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, x, gdim, gstr, box, ones, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_32B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return HARP_ERR_CUDA;
     }
-    const int n_row_tiles = (int)((n_rows + kRows - 1) / kRows);
-    for (const TmPass &ps : tp->pass[transpose ? 1 : 0]) {
-        TmParams prm;
-        prm.frags = ps.d_frags;
-        prm.n_row_tiles = n_row_tiles;
-        prm.n_col_tiles = ps.n_col_tiles;
-        prm.lo_count = ps.lo_count;
-        prm.err = tp->d_err;
-        const int64_t n_tiles = (int64_t)n_row_tiles * ps.n_col_tiles;
-        const int grid = (int)std::min<int64_t>(n_tiles, tp->n_sm);
-        prm.tiles_per_cta = (int)((n_tiles + grid - 1) / grid);
-        const int nph = ps.k1 < 0 ? 1 : 2;
-        const size_t smem = 1024 + (size_t)kNBuf * kTileBytes + 2 * (size_t)nph * kFragBytes;
-        cudaError_t e = cudaErrorInvalidValue;
-        const CUtensorMap &map = ps.fmt == FMT_C ? map_c : map_s;
-        if (ps.fmt == FMT_C && ps.k0 == TM_I && ps.k1 == TM_O) e = launch_one<FMT_C, TM_I, TM_O, 0>(map, prm, grid, smem, stream);
-        else if (ps.fmt == FMT_C && ps.k0 == TM_O && ps.k1 == TM_I) e = launch_one<FMT_C, TM_O, TM_I, 0>(map, prm, grid, smem, stream);
-        else if (ps.fmt == FMT_C && ps.k0 == TM_O && ps.k1 < 0) e = launch_one<FMT_C, TM_O, -1, 0>(map, prm, grid, smem, stream);
-        else if (ps.fmt == FMT_S && ps.k0 == TM_O && ps.k1 < 0 && !ps.xpose) e = launch_one<FMT_S, TM_O, -1, 0>(map, prm, grid, smem, stream);
-        else if (ps.fmt == FMT_S && ps.k0 == TM_O && ps.k1 < 0 && ps.xpose) e = launch_one<FMT_S, TM_O, -1, 1>(map, prm, grid, smem, stream);
-        else if (ps.fmt == FMT_S && ps.k0 == TM_I && ps.k1 < 0 && ps.xpose) e = launch_one<FMT_S, TM_I, -1, 1>(map, prm, grid, smem, stream);
-        if (e != cudaSuccess) return HARP_ERR_CUDA;
-        g_harp_launches.fetch_add(1, std::memory_order_relaxed);
-    }
     return HARP_OK;
+}
+
+harp_status_t run_pass(const TmPlan *tp, const TmPass &ps, const CUtensorMap &map, int64_t n_rows, cudaStream_t stream) {
+    const int n_row_tiles = (int)((n_rows + kRows - 1) / kRows);
+    TmParams prm;
+    prm.frags = ps.d_frags;
+    prm.n_row_tiles = n_row_tiles;
+    prm.n_col_tiles = ps.n_col_tiles;
+    prm.lo_count = ps.lo_count;
+    prm.err = tp->d_err;
+    const int64_t n_tiles = (int64_t)n_row_tiles * ps.n_col_tiles;
+    const int grid = (int)std::min<int64_t>(n_tiles, tp->n_sm);
+    prm.tiles_per_cta = (int)((n_tiles + grid - 1) / grid);
+    const int nph = ps.k1 < 0 ? 1 : 2;
+    const size_t smem = 1024 + (size_t)kNBuf * kTileBytes + 2 * (size_t)nph * kFragBytes;
+    cudaError_t e = cudaErrorInvalidValue;
+    if (ps.fmt == FMT_C && ps.k0 == TM_I && ps.k1 == TM_O) e = launch_one<FMT_C, TM_I, TM_O, 0>(map, prm, grid, smem, stream);
+    else if (ps.fmt == FMT_C && ps.k0 == TM_O && ps.k1 == TM_I) e = launch_one<FMT_C, TM_O, TM_I, 0>(map, prm, grid, smem, stream);
+    else if (ps.fmt == FMT_C && ps.k0 == TM_O && ps.k1 < 0) e = launch_one<FMT_C, TM_O, -1, 0>(map, prm, grid, smem, stream);
+    else if (ps.fmt == FMT_S && ps.k0 == TM_O && ps.k1 < 0 && !ps.xpose) e = launch_one<FMT_S, TM_O, -1, 0>(map, prm, grid, smem, stream);
+    else if (ps.fmt == FMT_S && ps.k0 == TM_O && ps.k1 < 0 && ps.xpose) e = launch_one<FMT_S, TM_O, -1, 1>(map, prm, grid, smem, stream);
+    else if (ps.fmt == FMT_S && ps.k0 == TM_I && ps.k1 < 0 && ps.xpose) e = launch_one<FMT_S, TM_I, -1, 1>(map, prm, grid, smem, stream);
+    if (e != cudaSuccess) return HARP_ERR_CUDA;
+    g_harp_launches.fetch_add(1, std::memory_order_relaxed);
+    return HARP_OK;
+}
+
+bool tm_args_ok(const void *x, int64_t n_rows, harp_dtype_t dtype) {
+    return dtype == HARP_BF16 && (reinterpret_cast<uintptr_t>(x) & 15u) == 0 && n_rows <= ((int64_t)1 << 30);
+}
+
+}  // namespace
+
+harp_status_t harp_tm_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype, int transpose,
+                            cudaStream_t stream) {
+    const TmPlan *tp = plan->tm;
+    if (!tp || tp->pass[0].empty() || !tm_args_ok(x, n_rows, dtype)) return HARP_ERR_UNSUPPORTED;
+    CUtensorMap map_c, map_s;
+    harp_status_t st = encode_maps(x, n_rows, plan->d, plan->d > 256, &map_c, &map_s);
+    for (const TmPass &ps : tp->pass[transpose ? 1 : 0])
+        if (st == HARP_OK) st = run_pass(tp, ps, ps.fmt == FMT_C ? map_c : map_s, n_rows, stream);
+    return st;
+}
+
+// Stages [0, harp_tm_slab_stages) only -- those below stride 256, with the sign diagonal -- on slabs of 256
+// contiguous coordinates (identity permutation): the lower pass of the two-pass paths for wide rows.
+int harp_tm_slab_stages(const harp_plan *plan) {
+    const TmPlan *tp = plan->tm;
+    if (!tp) return 0;
+    if (tp->has_slab) return tp->slab_stages;
+    return 0;
+}
+
+harp_status_t harp_tm_slab_apply(const harp_plan *plan, void *x, int64_t n_rows, harp_dtype_t dtype, int transpose,
+                                 cudaStream_t stream) {
+    const TmPlan *tp = plan->tm;
+    if (!tp || !tp->has_slab || !tm_args_ok(x, n_rows, dtype)) return HARP_ERR_UNSUPPORTED;
+    CUtensorMap map_c, map_s;
+    const harp_status_t st = encode_maps(x, n_rows, plan->d, false, &map_c, &map_s);
+    if (st != HARP_OK) return st;
+    return run_pass(tp, tp->slab[transpose ? 1 : 0], map_c, n_rows, stream);
 }
 
 // Copies the per-section cycle counters to out[16] (zeros unless built with -DHARP_TM_TIMING) and

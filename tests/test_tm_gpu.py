@@ -97,3 +97,23 @@ def test_cfg2_full_rows_sampled():
         x64 = promote(xh[rows], "bf16")
         want = orc.transpose(oplan, x64) if transpose else orc.forward(oplan, x64)
         assert orc.rel_err_rows(got[rows], want) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("transpose", [False, True])
+@pytest.mark.parametrize("cfg", [3, 4])
+def test_wide_rows_take_the_slab_pass(cfg, transpose):
+    """cfg3 (2^8 x 43) and cfg4 (16, 16, 8, 7): the stages below stride 256 run in the tensor-memory kernel,
+    the rest in the column-group kernels; 1300 rows (ten full 128-row tiles and a ragged one), every
+    element against the oracle."""
+    w = wl.config(cfg)
+    spec, data = w.plans["q"], w.data["x"]
+    plan = harp.plan_from_spec(spec)
+    oplan = orc.OraclePlan.from_spec(spec)
+    xh = data.rows(0, 1300)
+    before = harp.harp_launch_count()
+    got, ok = gpu_apply(plan, xh, "bf16", transpose=transpose)
+    assert ok and harp.harp_plan_error_word(plan) == 0
+    assert harp.harp_launch_count() - before == 2
+    x64 = promote(xh, "bf16")
+    want = orc.transpose(oplan, x64) if transpose else orc.forward(oplan, x64)
+    assert orc.rel_err_rows(got, want) <= TOL["bf16"]
