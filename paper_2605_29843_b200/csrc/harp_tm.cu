@@ -31,7 +31,7 @@ constexpr int kRows = 128;               // rows per tile = lanes of tensor memo
 constexpr int kTileBytes = 65536;        // 128 rows x 256 bf16
 constexpr int kNBuf = 3;                 // tile buffers in shared memory (ring; output staged in place)
 constexpr int kFragBytes = 8192;         // 16 blocks x 16 x 16 bf16 per phase
-constexpr int kThreads = 384;            // 12 warps: producer, MMA, store, idle, 2 x 4 epilogue
+constexpr int kThreads = 384;            // 12 warps: producer, MMA (chunk 0), store, MMA (chunk 1), 2 x 4 epilogue
 constexpr uint32_t kSpin = 1u << 22;     // limit of every wait
 constexpr int TM_I = 0, TM_O = 1;        // a phase contracts the inner (e) or the outer (q) index
 constexpr int FMT_C = 0, FMT_S = 1;      // contiguous 256 coordinates / 16 segments of 16
@@ -137,7 +137,7 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
     constexpr bool CROSS_OUT = (KLAST == TM_O) != (XPOSE != 0);
 
     extern __shared__ unsigned char smem_raw[];
-    __shared__ __align__(8) uint64_t bars[3 * kNBuf + 3];
+    __shared__ __align__(8) uint64_t bars[3 * kNBuf + 5];
     __shared__ uint32_t tmem_base_s;
     __shared__ int dead_s;
 
@@ -147,8 +147,9 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
     const uint32_t bar_full = smem_u32(&bars[0]);                  // + 8 b
     const uint32_t bar_empty = smem_u32(&bars[kNBuf]);
     const uint32_t bar_out = smem_u32(&bars[2 * kNBuf]);
-    const uint32_t bar_a = smem_u32(&bars[3 * kNBuf]);
-    const uint32_t bar_d = smem_u32(&bars[3 * kNBuf + 1]);         // two of them
+    const uint32_t bar_a = smem_u32(&bars[3 * kNBuf]);             // two: A of the first phase, per warpgroup
+    const uint32_t bar_a2 = smem_u32(&bars[3 * kNBuf + 2]);        // A of the second phase (both warpgroups)
+    const uint32_t bar_d = smem_u32(&bars[3 * kNBuf + 3]);         // two: D chunk of a warpgroup
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -157,7 +158,9 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
             mbar_init(bar_empty + 8 * b, 1);
             mbar_init(bar_out + 8 * b, 256);
         }
-        mbar_init(bar_a, 256);
+        mbar_init(bar_a, 128);
+        mbar_init(bar_a + 8, 128);
+        mbar_init(bar_a2, 256);
         mbar_init(bar_d, 1);
         mbar_init(bar_d + 8, 1);
         dead_s = 0;
@@ -226,9 +229,10 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
                         if (mbar_try(bar_full + 8 * (int)(k % kNBuf), (uint32_t)((k / kNBuf) & 1))) break;
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issue ----------------
+    } else if (warp == 1 || warp == 3) {
+        // ---------------- MMA issue: warp 1 for chunk 0 (blocks 0-7), warp 3 for chunk 1 ----------------
         if (lane == 0) {
+            const int g = warp == 1 ? 0 : 1;
             const uint32_t idesc = instr_desc(128, 16);
             int cur_col = -1, slot = 1;
             uint32_t ua = 0;
@@ -240,30 +244,31 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
 #pragma unroll
                 for (int ph = 0; ph < NPH; ++ph) {
                     TM_T(c0);
-                    if (!wait(bar_a, ua & 1, 3)) { ok = false; break; }
+                    // the first phase needs this chunk's own blocks of A (written by its warpgroup), the second
+                    // the whole of A (pairs from both warpgroups)
+                    if (!wait(ph == 0 ? bar_a + 8 * g : bar_a2, ua & 1, 3)) { ok = false; break; }
                     TM_T(c1);
                     TM_ACC(3, c0, c1);
-                    ++ua;
                     tc_fence_after();
                     const uint32_t a_col = ph == 0 ? kColA1 : kColA2;
                     const uint32_t fbase = frag0 + slot * (NPH * kFragBytes) + ph * kFragBytes;
 #pragma unroll
-                    for (int g = 0; g < 2; ++g) {
-#pragma unroll
-                        for (int blk = 0; blk < 8; ++blk) {
-                            const int c = g * 8 + blk;
-                            mma_ts(tmem + kColD + c * 16, tmem + a_col + c * 8, smem_desc(fbase + c * 512, 128, 256), idesc);
-                        }
-                        mma_commit(bar_d + 8 * g);
+                    for (int blk = 0; blk < 8; ++blk) {
+                        const int c = g * 8 + blk;
+                        mma_ts(tmem + kColD + c * 16, tmem + a_col + c * 8, smem_desc(fbase + c * 512, 128, 256), idesc);
                     }
+                    mma_commit(bar_d + 8 * g);
                     TM_T(c2);
                     TM_ACC(4, c1, c2);
                 }
+                ++ua;
                 if (!ok) break;
             }
 #ifdef HARP_TM_TIMING
-            atomicAdd((unsigned long long *)&g_tm_timing[3], (unsigned long long)acc[3]);
-            atomicAdd((unsigned long long *)&g_tm_timing[4], (unsigned long long)acc[4]);
+            if (g == 0) {
+                atomicAdd((unsigned long long *)&g_tm_timing[3], (unsigned long long)acc[3]);
+                atomicAdd((unsigned long long *)&g_tm_timing[4], (unsigned long long)acc[4]);
+            }
 #endif
         }
     } else if (warp == 2) {
@@ -344,7 +349,7 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
             }
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(bar_a);
+            mbar_arrive(bar_a + 8 * g);
             TM_T(e2);
             TM_ACC(8, e1, e2);
             if (!wait(bar_d + 8 * g, ud & 1, 6)) break;
@@ -356,6 +361,9 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
                 // --- between the phases: D (fp32) -> A of the other index (bf16 pairs over neighbouring blocks) ---
                 uint32_t p[64];
                 pack_cross(tlane + kColD + 128 * g, p);
+                // A of the second phase is shared by both chunks: the other chunk's second-phase products of the
+                // tile before must be complete, which that tile's out barrier implies (its warpgroup read them)
+                if (i > 0 && !wait(bar_out + 8 * (int)((i - 1) % kNBuf), (uint32_t)(((i - 1) / kNBuf) & 1), 8)) break;
 #pragma unroll
                 for (int j = 0; j < 16; ++j) {
                     const uint32_t v4[4] = {p[j * 4 + 0], p[j * 4 + 1], p[j * 4 + 2], p[j * 4 + 3]};
@@ -363,7 +371,7 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
                 }
                 tmem_wait_st();
                 tc_fence_before();
-                mbar_arrive(bar_a);
+                mbar_arrive(bar_a2);
                 TM_T(e4);
                 TM_ACC(10, e3, e4);
                 if (!wait(bar_d + 8 * g, ud & 1, 7)) break;
