@@ -1,3 +1,15 @@
+// Measured on B200 while this file was written (a probe program, one run each):
+//  * shared-memory operand descriptor, K-major, no swizzle: leading byte offset = step between the 8-row x
+//    16-byte core matrices along K, stride byte offset = step along N/M (a 16 x 16 bf16 block stored as
+//    [n/8][k/8][n%8][k%8]: lbo 128, sbo 256); the other assignment gives a wrong product;
+//  * A operand in tensor memory: row i in lane i, two bf16 per 32-bit column, even k in the low half;
+//  * one tcgen05.mma with M = 128, K = 16 and A in tensor memory costs about 47 cycles for N = 16, 32 or 64
+//    (65 for N = 128);
+//  * a tiled tensor map with the 128-byte swizzle places box rows shorter than 128 bytes at a 128-byte pitch
+//    in shared memory (a 32-byte inner box overruns a buffer sized for packed rows); the 32-byte swizzle packs
+//    them: byte L of the packed image lands at L ^ (((L >> 7) & 1) << 4);
+//  * 128-byte swizzle, 128-byte rows: 16-byte chunk c of row r lands at r * 128 + ((c ^ (r & 7)) << 4).
+//
 // PTX wrappers of the Blackwell-only machinery used by harp_tm.cu: mbarriers with bounded waits,
 // tiled bulk tensor copies (TMA, never multicast), tensor memory allocation, tcgen05.mma with the A
 // operand in tensor memory, and the tensor-memory load/store forms.
