@@ -310,46 +310,51 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
         const uint32_t tlane = tmem + ((uint32_t)((warp & 3) << 5) << 16);
         uint32_t ud = 0;
         TM_DECL;
+        // row r of the tile in buffer `src` -> this warpgroup's half of the first phase's A operand
+        auto row_to_a1 = [&](uint32_t src) {
+            uint32_t a[64];
+            if (K0 == TM_I) {
+                // blocks q = 8g .. 8g+7, K = e: the row's own order
+#pragma unroll
+                for (int beta = 0; beta < 8; ++beta)
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const uint4 v = lds128(src + chunk_off<FMT>(r, 8 * g + beta, h));
+                        a[beta * 8 + h * 4 + 0] = v.x; a[beta * 8 + h * 4 + 1] = v.y;
+                        a[beta * 8 + h * 4 + 2] = v.z; a[beta * 8 + h * 4 + 3] = v.w;
+                    }
+            } else {
+                // blocks e = 8g .. 8g+7, K = q: pair (q = 2m, 2m+1) at fixed e
+                uint32_t c[16][4];
+#pragma unroll
+                for (int q = 0; q < 16; ++q) {
+                    const uint4 v = lds128(src + chunk_off<FMT>(r, q, g));
+                    c[q][0] = v.x; c[q][1] = v.y; c[q][2] = v.z; c[q][3] = v.w;
+                }
+#pragma unroll
+                for (int eps = 0; eps < 8; ++eps)
+#pragma unroll
+                    for (int m = 0; m < 8; ++m)
+                        a[eps * 8 + m] = prmt(c[2 * m][eps >> 1], c[2 * m + 1][eps >> 1], (eps & 1) ? 0x7632u : 0x5410u);
+            }
+            tmem_st64(tlane + kColA1 + 64 * g, a);
+        };
         for (int64_t t = t_begin; t < t_end; ++t) {
             const int64_t i = t - t_begin;
             const int b = (int)(i % kNBuf);
             const uint32_t buf = buf0 + b * kTileBytes;
             TM_T(e0);
-            if (!wait(bar_full + 8 * b, (uint32_t)((i / kNBuf) & 1), 5)) break;
+            // two-phase passes fetch the next tile's row early (see below); then this tile's A is already there
+            const bool a1_done = NPH == 2 && i > 0;
+            if (!a1_done && !wait(bar_full + 8 * b, (uint32_t)((i / kNBuf) & 1), 5)) break;
             TM_T(e1);
             TM_ACC(7, e0, e1);
-            // --- row from shared memory to the A operand of the first phase ---
-            {
-                uint32_t a[64];
-                if (K0 == TM_I) {
-                    // blocks q = 8g .. 8g+7, K = e: the row's own order
-#pragma unroll
-                    for (int beta = 0; beta < 8; ++beta)
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            const uint4 v = lds128(buf + chunk_off<FMT>(r, 8 * g + beta, h));
-                            a[beta * 8 + h * 4 + 0] = v.x; a[beta * 8 + h * 4 + 1] = v.y;
-                            a[beta * 8 + h * 4 + 2] = v.z; a[beta * 8 + h * 4 + 3] = v.w;
-                        }
-                } else {
-                    // blocks e = 8g .. 8g+7, K = q: pair (q = 2m, 2m+1) at fixed e
-                    uint32_t c[16][4];
-#pragma unroll
-                    for (int q = 0; q < 16; ++q) {
-                        const uint4 v = lds128(buf + chunk_off<FMT>(r, q, g));
-                        c[q][0] = v.x; c[q][1] = v.y; c[q][2] = v.z; c[q][3] = v.w;
-                    }
-#pragma unroll
-                    for (int eps = 0; eps < 8; ++eps)
-#pragma unroll
-                        for (int m = 0; m < 8; ++m)
-                            a[eps * 8 + m] = prmt(c[2 * m][eps >> 1], c[2 * m + 1][eps >> 1], (eps & 1) ? 0x7632u : 0x5410u);
-                }
-                tmem_st64(tlane + kColA1 + 64 * g, a);
+            if (!a1_done) {
+                row_to_a1(buf);
+                tmem_wait_st();
+                tc_fence_before();
+                mbar_arrive(bar_a + 8 * g);
             }
-            tmem_wait_st();
-            tc_fence_before();
-            mbar_arrive(bar_a + 8 * g);
             TM_T(e2);
             TM_ACC(8, e1, e2);
             if (!wait(bar_d + 8 * g, ud & 1, 6)) break;
@@ -357,6 +362,7 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
             tc_fence_after();
             TM_T(e3);
             TM_ACC(9, e2, e3);
+            bool next_a1 = false;
             if (NPH == 2) {
                 // --- between the phases: D (fp32) -> A of the other index (bf16 pairs over neighbouring blocks) ---
                 uint32_t p[64];
@@ -374,6 +380,17 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
                 mbar_arrive(bar_a2);
                 TM_T(e4);
                 TM_ACC(10, e3, e4);
+                // While the second phase's products run: the next tile's row into this warpgroup's half of the
+                // first phase's A (its own first-phase products of this tile are complete, nobody else reads that
+                // half).  The barrier that releases the next tile's first phase is arrived on further down, once
+                // this tile's accumulators have been read.
+                if (t + 1 < t_end) {
+                    const int64_t i2 = i + 1;
+                    if (!wait(bar_full + 8 * (int)(i2 % kNBuf), (uint32_t)((i2 / kNBuf) & 1), 5)) break;
+                    row_to_a1(buf0 + (int)(i2 % kNBuf) * kTileBytes);
+                    tmem_wait_st();
+                    next_a1 = true;
+                }
                 if (!wait(bar_d + 8 * g, ud & 1, 7)) break;
                 ++ud;
                 tc_fence_after();
@@ -385,10 +402,15 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
             if (CROSS_OUT) {
                 uint32_t p[64];
                 pack_cross(tlane + kColD + 128 * g, p);
+                if (next_a1) {                      // accumulators read: the next tile's first phase may overwrite them
+                    tc_fence_before();
+                    mbar_arrive(bar_a + 8 * g);
+                }
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
                     sts128(buf + chunk_off<FMT>(r, j, g), p[j * 4 + 0], p[j * 4 + 1], p[j * 4 + 2], p[j * 4 + 3]);
             } else {
+                uint32_t o4[16][4];
 #pragma unroll
                 for (int pair = 0; pair < 4; ++pair) {
                     uint32_t d[32];
@@ -399,13 +421,18 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
                             const int o = bb * 16 + h * 8;
-                            sts128(buf + chunk_off<FMT>(r, 8 * g + 2 * pair + bb, h),
-                                   pack_bf16x2(__uint_as_float(d[o + 0]), __uint_as_float(d[o + 1])),
-                                   pack_bf16x2(__uint_as_float(d[o + 2]), __uint_as_float(d[o + 3])),
-                                   pack_bf16x2(__uint_as_float(d[o + 4]), __uint_as_float(d[o + 5])),
-                                   pack_bf16x2(__uint_as_float(d[o + 6]), __uint_as_float(d[o + 7])));
+#pragma unroll
+                            for (int u = 0; u < 4; ++u)
+                                o4[pair * 4 + bb * 2 + h][u] = pack_bf16x2(__uint_as_float(d[o + 2 * u]), __uint_as_float(d[o + 2 * u + 1]));
                         }
                 }
+                if (next_a1) {
+                    tc_fence_before();
+                    mbar_arrive(bar_a + 8 * g);
+                }
+#pragma unroll
+                for (int k = 0; k < 16; ++k)        // chunk (q = 8g + k/2, h = k & 1)
+                    sts128(buf + chunk_off<FMT>(r, 8 * g + (k >> 1), k & 1), o4[k][0], o4[k][1], o4[k][2], o4[k][3]);
             }
             tc_fence_before();
             fence_async_smem();
