@@ -305,6 +305,13 @@ harp_status_t harp_apply_host(harp_plan_t *plan, void *x_host, int64_t n_rows,
  * code naming the wait otherwise, -1 for NULL or a failed copy.  Synchronises with the device. */
 int32_t harp_plan_error_word(const harp_plan_t *plan);
 
+/* Per-section cycle counters of the tensor-memory kernels and of the whole-row kernel, for profiling
+ * notes.  They count only in a library built with HARP_TM_TIMING=1 / HARP_FAST_TIMING=1 in the
+ * environment of the build step (clock reads at section boundaries, summed over CTAs; slot 0 = tiles);
+ * otherwise the sixteen slots read zero.  out HOST int64[16]; reset != 0 clears them.  0 on success. */
+int32_t harp_debug_tm_timing(int64_t *out, int32_t reset);
+int32_t harp_debug_fast_timing(int64_t *out, int32_t reset);
+
 /* Number of kernels this library has launched in the calling process (all plans). */
 int64_t harp_launch_count(void);
 

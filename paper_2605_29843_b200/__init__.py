@@ -99,6 +99,25 @@ def status_string(status: int) -> str:
     return lib().harp_status_string(int(status)).decode()
 
 
+def _debug_timing(fn_name: str, reset: bool):
+    L = lib()
+    fn = getattr(L, fn_name)
+    fn.restype = ctypes.c_int32
+    fn.argtypes = [ctypes.c_void_p, ctypes.c_int32]
+    out = (ctypes.c_int64 * 16)()
+    if fn(out, 1 if reset else 0) != 0:
+        raise HarpError(10, fn_name)
+    return list(out)
+
+
+def harp_debug_tm_timing(reset: bool = True):
+    return _debug_timing("harp_debug_tm_timing", reset)
+
+
+def harp_debug_fast_timing(reset: bool = True):
+    return _debug_timing("harp_debug_fast_timing", reset)
+
+
 def harp_plan_error_word(plan) -> int:
     return int(lib().harp_plan_error_word(plan.handle if hasattr(plan, "handle") else plan))
 

@@ -36,6 +36,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         cmd += ["-Xptxas", "-v"]
     if os.environ.get("HARP_TM_TIMING"):          # per-section cycle counters in the tensor-memory kernels
         cmd += ["-DHARP_TM_TIMING"]
+    if os.environ.get("HARP_FAST_TIMING"):        # ... and in the whole-row kernel
+        cmd += ["-DHARP_FAST_TIMING"]
     cmd += sources() + ["-o", LIB]
     subprocess.check_call(cmd)
     return LIB

@@ -81,6 +81,16 @@ struct FastParams {
     PhaseDesc ph[kMaxPhases];
 };
 
+// Per-section cycle counters of the whole-row kernel (build with -DHARP_FAST_TIMING): thread 0 of every CTA
+// reads the clock after the barrier that ends a section; sums over CTAs and tiles.
+//  0 tiles | 1 copy in | 2 .. 2+kMaxPhases-1 phase k | 10 copy out
+__device__ long long g_fast_timing[16];
+#ifdef HARP_FAST_TIMING
+#define FAST_MARK(slot) do { if (threadIdx.x == 0) { const long long now_ = clock64(); tacc[slot] += now_ - tlast; tlast = now_; } } while (0)
+#else
+#define FAST_MARK(slot) do { } while (0)
+#endif
+
 // fragments of one item (eight blocks, one uint4 per lane and block): from tensor memory when the
 // phase is kept there, else from global memory
 __device__ __forceinline__ void load_frag8(uint4 (&bf)[8], const uint4 *bp, bool in_tm, uint32_t tm_addr) {
@@ -214,8 +224,14 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
         const long long wait = (long long)(blockIdx.x % 3) * stagger, t0 = clock64();
         while (clock64() - t0 < wait) { }
     }
+#ifdef HARP_FAST_TIMING
+    long long tacc[16] = {0}, tlast = clock64();
+#endif
     for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
         const int64_t row0 = tile * kTileRows;
+#ifdef HARP_FAST_TIMING
+        if (threadIdx.x == 0) { tacc[0] += 1; tlast = clock64(); }
+#endif
         // rows past the end of the batch are computed on a copy of the last row and never stored
         const int64_t last = n_rows - 1;
         c.okA = row0 + c.g < n_rows;
@@ -238,6 +254,7 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
             cp_async_wait_all();
             __syncthreads();
         }
+        FAST_MARK(1);
 
         for (int p = 0; p < P.n_phases; ++p) {
             const PhaseDesc &ph = P.ph[p];
@@ -383,6 +400,7 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
                 }
             }
             __syncthreads();
+            FAST_MARK(2 + p);
         }
 
         if (P.copy_out >= 0) {
@@ -397,7 +415,13 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
             }
             __syncthreads();
         }
+        FAST_MARK(10);
     }
+#ifdef HARP_FAST_TIMING
+    if (threadIdx.x == 0)
+        for (int k = 0; k < 16; ++k)
+            if (tacc[k]) atomicAdd((unsigned long long *)&g_fast_timing[k], (unsigned long long)tacc[k]);
+#endif
     if (P.tm_mask) {
         harp_tm::tc_fence_before();
         __syncthreads();
@@ -990,6 +1014,18 @@ harp_status_t harp_fast_build(harp_plan *plan) {
         return st;
     }
     return HARP_OK;
+}
+
+// Copies the per-section cycle counters to out[16] (zeros unless built with -DHARP_FAST_TIMING) and clears
+// them if asked.
+extern "C" int32_t harp_debug_fast_timing(int64_t *out, int32_t reset) {
+    if (!out) return -1;
+    if (cudaMemcpyFromSymbol(out, g_fast_timing, sizeof(long long) * 16) != cudaSuccess) return -1;
+    if (reset) {
+        const long long zero[16] = {0};
+        if (cudaMemcpyToSymbol(g_fast_timing, zero, sizeof(zero)) != cudaSuccess) return -1;
+    }
+    return 0;
 }
 
 void harp_fast_destroy(harp_plan *plan) {
