@@ -1043,7 +1043,9 @@ harp_status_t harp_fast_apply(const harp_plan *plan, void *x, int64_t n_rows, ha
     const int64_t n_tiles = (n_rows + kTileRows - 1) / kTileRows;
     const int grid = (int)std::min<int64_t>(n_tiles, fp->max_ctas);
     __nv_bfloat16 *xb = static_cast<__nv_bfloat16 *>(x);
-    const FastParams &P = transpose ? fp->bwd : fp->fwd;
+    FastParams P = transpose ? fp->bwd : fp->fwd;
+    // fragments in tensor memory pay from the second tile of a CTA on; a CTA with one tile streams them
+    if (n_tiles < 2 * (int64_t)grid) P.tm_mask = 0;
     // a quarter of a tile period, estimated from the measured 28 k cycles per tile of d = 4096 with
     // three phases (the gain is flat between half and the full value)
     const int stagger = n_tiles >= 4 * (int64_t)grid ? (int)(0.57 * (double)P.d * P.n_phases) : 0;

@@ -26,14 +26,16 @@ def test_round_trip_and_norm_drift(cfg, n_rows):
     torch.cuda.synchronize()
     y = to_host_f64(x)
     nx, ny = np.linalg.norm(x64, axis=1), np.linalg.norm(y, axis=1)
-    # Q is orthogonal: the norm of every row survives, up to the roundings (each at most 2^-9 relative per
-    # coordinate and independent, so far below 2^-8 on the norm)
-    assert np.max(np.abs(ny / nx - 1.0)) <= 2e-3
+    # Q is orthogonal: the norm of every row survives, up to the roundings.  One rounding moves a
+    # coordinate by at most 2^-9 of its size, hence the norm by at most 2^-9 (reached when one coordinate
+    # carries the row, as in the heavy-tailed rows); at most four roundings per coordinate on these plans
+    drift = float(np.max(np.abs(ny / nx - 1.0)))
+    assert drift <= 4 * 2.0 ** -9, drift
     harp.apply_(plan, x, transpose=True)
     torch.cuda.synchronize()
     back = to_host_f64(x)
     # forward then transpose is the identity: two applies' worth of error, relative to the row norm
-    err = np.max(np.max(np.abs(back - x64), axis=1) / nx)
-    assert err <= 2 * TOL["bf16"]
+    err = float(np.max(np.max(np.abs(back - x64), axis=1) / nx))
+    assert err <= 2 * TOL["bf16"], err
     # and the error does not pile up on the outlier channels' rows more than elsewhere: same bound per row
     assert harp.harp_plan_error_word(plan) == 0
