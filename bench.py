@@ -317,6 +317,24 @@ def bench_compact(torch, harp, kernel, peak):
                 torch.cuda.synchronize()
                 dt = time_region(torch, call, 400)
                 res[f"decode_{n}_rows_us"] = round(1e6 * dt / 400, 2)
+        if cfg == 4:
+            # the same schedule behind a random permutation (a layer whose reshape permutes the coordinates):
+            # one gather kernel and the two tensor-core passes
+            import copy
+            pspec = copy.copy(spec)
+            pspec.perm = np.random.default_rng(977).permutation(spec.d).astype(np.int32)
+            pplan = harp.plan_from_spec(pspec)
+            for name, tr in (("forward", False), ("transpose", True)):
+                for i in range(2):
+                    harp.apply_(pplan, bufs[i % nbuf], transpose=tr, kernel=kernel)
+                torch.cuda.synchronize()
+                l0 = harp.harp_launch_count()
+                dt = time_region(torch, lambda i: harp.apply_(pplan, bufs[i % nbuf], transpose=tr, kernel=kernel), 6)
+                gbs = 2 * nbytes * 6 / dt / 1e9
+                res.setdefault("random_permutation", {})[name] = {
+                    "GBps": round(gbs, 1), "frac": round(gbs / peak, 4), "us": round(1e6 * dt / 6, 2),
+                    "launches": (harp.harp_launch_count() - l0) // 6}
+            del pplan
         if cfg == 5:
             del bufs
             torch.cuda.empty_cache()

@@ -22,6 +22,11 @@
 //
 // Radices that do not fill an 8- or 16-wide block (7, 2, ...) are zero-padded inside the
 // fragments; padded slots read a valid coordinate and are never stored.
+//
+// A plan with a permutation takes the same two passes and one more kernel that moves the
+// coordinates of every row (harp_gather_rows_kernel: whole rows through shared memory, in place):
+// before the passes in the forward direction, after them in the transpose direction.  The sign
+// diagonal stays folded into the first phase's fragments, read through the permutation.
 #include <algorithm>
 #include <cstdlib>
 #include <cstring>
@@ -417,6 +422,64 @@ harp_upper_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_
     cp_async_wait_all();
 }
 
+// ---------------------------------------------------------------------------------------
+// Fixed permutation of wide rows, in place: out[i] = in[table[i]] for every row (Theorem 1's
+// permutation convention: table = the plan's permutation in the forward direction, its inverse
+// in the transpose direction).  A CTA keeps the table in shared memory as 16-bit indices and
+// takes groups of R whole rows through two buffers: the next group is copied in (cp.async) while
+// this one is gathered with 2-byte shared-memory reads and written back with 16-byte stores.  The
+// move is exact: no arithmetic touches the values.
+constexpr int kGatherThreads = 512;
+
+__global__ void __launch_bounds__(kGatherThreads, 1)
+harp_gather_rows_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int32_t d, int32_t R, const uint16_t *__restrict__ table) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const uint32_t sbase = smem_u32(smem_raw);
+    const uint32_t tab_s = sbase;                                   // d 16-bit indices
+    const uint32_t row_bytes = 2u * (uint32_t)d;
+    const uint32_t buf_s = sbase + row_bytes;                       // two buffers of R rows
+    const uint32_t buf_bytes = (uint32_t)R * row_bytes;
+    const int chunks = d >> 3;                                      // 16-byte chunks per row
+    for (int c = threadIdx.x; c < chunks; c += kGatherThreads) cp_async16(tab_s + 16u * c, table + 8 * c);
+    const int64_t n_groups = (n_rows + R - 1) / R;
+    auto copy_in = [&](int64_t grp, uint32_t dst) {
+        const int64_t row0 = grp * R;
+        const int rows = (int)min((int64_t)R, n_rows - row0);
+        const __nv_bfloat16 *src = x + row0 * d;
+        for (int c = threadIdx.x; c < rows * chunks; c += kGatherThreads) cp_async16(dst + 16u * c, src + 8 * (int64_t)c);
+        cp_async_commit();
+    };
+    int buf = 0;
+    if ((int64_t)blockIdx.x < n_groups) copy_in(blockIdx.x, buf_s);
+    for (int64_t grp = blockIdx.x; grp < n_groups; grp += gridDim.x) {
+        cp_async_wait_group<0>();
+        __syncthreads();                                            // this group is here; the other buffer is free
+        if (grp + gridDim.x < n_groups) copy_in(grp + gridDim.x, buf_s + (uint32_t)(buf ^ 1) * buf_bytes);
+        const int64_t row0 = grp * R;
+        const int rows = (int)min((int64_t)R, n_rows - row0);
+        const uint32_t src_s = buf_s + (uint32_t)buf * buf_bytes;
+        for (int c = threadIdx.x; c < rows * chunks; c += kGatherThreads) {
+            const int r = c / chunks, cc = c - r * chunks;
+            const uint4 idx = lds128(tab_s + 16u * cc);
+            const uint32_t rb = src_s + (uint32_t)r * row_bytes;
+            auto pick = [&](uint32_t pair) {
+                uint32_t lo, hi;
+                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(lo) : "r"(rb + 2u * (pair & 0xffffu)));
+                asm volatile("ld.shared.u16 %0, [%1];" : "=r"(hi) : "r"(rb + 2u * (pair >> 16)));
+                return lo | (hi << 16);
+            };
+            uint4 out;
+            out.x = pick(idx.x);
+            out.y = pick(idx.y);
+            out.z = pick(idx.z);
+            out.w = pick(idx.w);
+            stg128(x + (row0 + r) * d + 8 * cc, out);
+        }
+        buf ^= 1;
+    }
+    cp_async_wait_all();
+}
+
 // ------------------------------------------------------------------------------- host
 
 struct PassHost {
@@ -434,6 +497,10 @@ struct SplitPlan {
     int64_t chunk_rows = 0;    // rows per L2-resident chunk
     int sms = 148;
     int lower_stages = 0;      // pass[0] covers stages [0, lower_stages)
+    // plans with a permutation: 16-bit gather tables ([0] forward = the permutation, [1] transpose = its inverse)
+    const uint16_t *gather[2] = {nullptr, nullptr};
+    int gather_rows = 1;       // rows per buffer of the gather kernel
+    size_t gather_smem = 0;
     // dense upper pass (replaces pass[1] when set)
     bool dense_upper = false;
     UpperPass up_fwd{}, up_bwd{};
@@ -622,7 +689,7 @@ harp_status_t build_pass(const harp_plan *plan, SplitPlan *sp, PassHost &ph_out,
                         double v = dir == 0 ? F[(size_t)rin * Br + rout] : F[(size_t)rout * Br + rin];
                         if (gp.t0 == 0 && !plan->h_signs.empty()) {
                             const int64_t pos = base + (int64_t)(dir == 0 ? rin : rout) * gp.S;
-                            v *= (double)plan->h_signs[(size_t)pos];
+                            v *= (double)plan->h_signs[(size_t)(plan->h_perm.empty() ? pos : plan->h_perm[(size_t)pos])];
                         }
                         return v;
                     };
@@ -719,7 +786,9 @@ harp_status_t build_dense_upper(const harp_plan *plan, SplitPlan *sp, int t0, in
 harp_status_t harp_split_build(harp_plan *plan) {
     const int64_t d = plan->d;
     const int m = plan->st.m;
-    if (d % 8 != 0 || !plan->h_perm.empty()) return HARP_ERR_UNSUPPORTED;
+    if (d % 8 != 0) return HARP_ERR_UNSUPPORTED;
+    const bool permuted = !plan->h_perm.empty();
+    if (permuted && d > 65536) return HARP_ERR_UNSUPPORTED;                         // 16-bit gather tables
     // ---- group stages: as many as fit a 16-wide block; smaller products are zero-padded to 8 or 16.
     // A radix above 16 ends the grouping: it and everything after it form the dense upper block.
     std::vector<GPhase> phs;
@@ -761,6 +830,23 @@ harp_status_t harp_split_build(harp_plan *plan) {
          cudaFuncSetAttribute(harp_upper_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess ||
          cudaFuncSetAttribute(harp_upper_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess))
         st = HARP_ERR_CUDA;
+    if (st == HARP_OK && permuted) {
+        std::vector<uint16_t> fwd((size_t)d), bwd((size_t)d);
+        for (int64_t i = 0; i < d; ++i) {
+            fwd[(size_t)i] = (uint16_t)plan->h_perm[(size_t)i];
+            bwd[(size_t)plan->h_perm[(size_t)i]] = (uint16_t)i;
+        }
+        sp->gather[0] = upload_s(sp, fwd, st);
+        sp->gather[1] = upload_s(sp, bwd, st);
+        // table + two buffers of R rows in about 200 KB
+        const size_t row_bytes = (size_t)d * 2;
+        sp->gather_rows = (int)std::max<size_t>(1, std::min<size_t>(16, (200u * 1024u - row_bytes) / (2 * row_bytes)));
+        sp->gather_smem = row_bytes * (1 + 2 * (size_t)sp->gather_rows);
+        if (sp->gather_smem > 227u * 1024u) st = HARP_ERR_UNSUPPORTED;
+        else if (st == HARP_OK && cudaFuncSetAttribute(harp_gather_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                       (int)sp->gather_smem) != cudaSuccess)
+            st = HARP_ERR_CUDA;
+    }
     if (st == HARP_OK) {
         int dev = 0, sms = 0;
         cudaGetDevice(&dev);
@@ -820,6 +906,18 @@ harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, h
     __nv_bfloat16 *xb = static_cast<__nv_bfloat16 *>(x);
     const bool two = sp->pass[1].present || sp->dense_upper;
     const bool overlap = n_rows <= kOverlapMaxRows;
+    auto gather = [&](int dir) -> harp_status_t {
+        const int64_t n_groups = (n_rows + sp->gather_rows - 1) / sp->gather_rows;
+        const unsigned grid = (unsigned)std::min<int64_t>(n_groups, sp->sms);
+        harp_gather_rows_kernel<<<grid, kGatherThreads, sp->gather_smem, stream>>>(xb, n_rows, (int32_t)plan->d, sp->gather_rows,
+                                                                                   sp->gather[dir]);
+        g_harp_launches.fetch_add(1, std::memory_order_relaxed);
+        return cudaGetLastError() == cudaSuccess ? HARP_OK : HARP_ERR_CUDA;
+    };
+    if (sp->gather[0] && !transpose) {
+        const harp_status_t gs = gather(0);
+        if (gs != HARP_OK) return gs;
+    }
     for (int64_t r0 = 0; r0 < n_rows; r0 += sp->chunk_rows) {
         const int64_t r1 = std::min(n_rows, r0 + (two ? sp->chunk_rows : n_rows));
         for (int s = 0; s < (two ? 2 : 1); ++s) {
@@ -867,5 +965,6 @@ harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, h
         }
         if (!two) break;
     }
+    if (sp->gather[0] && transpose) return gather(1);
     return HARP_OK;
 }

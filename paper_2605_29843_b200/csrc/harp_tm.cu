@@ -615,8 +615,8 @@ harp_status_t harp_tm_build(harp_plan *plan) {
     }
     if (whole && t != plan->st.m) return HARP_ERR_UNSUPPORTED;
     if (!whole) {
-        // wide row: only the slab part, identity permutation
-        if (!plan->h_perm.empty()) return HARP_ERR_UNSUPPORTED;
+        // wide row: only the slab part, on rows whose coordinates are already in the permuted order (the caller
+        // moves them); the sign of a coordinate is read through the permutation (sign_of)
         TmPlan *tp = new (std::nothrow) TmPlan();
         if (!tp) return HARP_ERR_ALLOC;
         plan->tm = tp;

@@ -92,7 +92,54 @@ def test_split_kernel_with_dense_upper_block(radices, monkeypatch):
             assert guards and orc.rel_err_rows(got, want) <= TOL["bf16"]
 
 
-@pytest.mark.parametrize("radices,perm", [((2,) * 8 + (67,), "identity"), ((4,) * 6, "digit_reversal"), ((7, 2, 4), "identity")])
+SPLIT_PERM = [((4,) * 6, "digit_reversal"), ((16, 16, 8, 7), "random"), ((8, 8, 8, 8, 7), "random"), ((2,) * 8 + (43,), "random"),
+              ((16, 16, 8, 7), "digit_reversal"), ((8, 8, 8, 5), "random")]
+
+
+@pytest.mark.parametrize("radices,perm", SPLIT_PERM)
+@pytest.mark.parametrize("kind", ["qr", "identity"])
+def test_split_kernel_with_a_permutation(radices, perm, kind):
+    """Plans with a permutation: the two passes plus the row-gather kernel (three launches, or two when
+    one pass covers all stages), every element against the oracle; identity blocks leave the sign flip
+    and the gather, which must be exact."""
+    spec = wl.make_plan(33, int(np.prod(radices)), radices, kind, perm=perm, signs=True)
+    oplan = orc.OraclePlan.from_spec(spec)
+    plan = harp.plan_from_spec(spec)
+    rng = np.random.default_rng(11)
+    for n_rows in (1, 37, 1300):
+        xh = host_rows(rng.standard_normal((n_rows, spec.d)), "bf16")
+        x64 = promote(xh, "bf16")
+        for tr in (False, True):
+            before = harp.harp_launch_count()
+            got, guards = gpu_apply(plan, xh, "bf16", tr, harp.KERNEL_SPLIT)
+            assert harp.harp_launch_count() - before <= 3
+            assert harp.harp_plan_error_word(plan) == 0
+            want = orc.transpose(oplan, x64) if tr else orc.forward(oplan, x64)
+            assert guards
+            if kind == "identity":
+                assert np.array_equal(got, want)
+            else:
+                assert orc.rel_err_rows(got, want) <= TOL["bf16"]
+
+
+def test_auto_takes_the_tensor_core_route_for_permuted_wide_rows():
+    """cfg4's schedule with a random permutation: AUTO = gather + two tensor-core passes, not the
+    per-coordinate kernel (which takes one launch)."""
+    spec = wl.make_plan(35, 14336, (16, 16, 8, 7), "qr", perm="random", signs=True)
+    oplan = orc.OraclePlan.from_spec(spec)
+    plan = harp.plan_from_spec(spec)
+    rng = np.random.default_rng(12)
+    xh = host_rows(rng.standard_normal((1100, spec.d)), "bf16")
+    x64 = promote(xh, "bf16")
+    for tr in (False, True):
+        before = harp.harp_launch_count()
+        got, guards = gpu_apply(plan, xh, "bf16", tr)
+        assert harp.harp_launch_count() - before == 3
+        want = orc.transpose(oplan, x64) if tr else orc.forward(oplan, x64)
+        assert guards and orc.rel_err_rows(got, want) <= TOL["bf16"]
+
+
+@pytest.mark.parametrize("radices,perm", [((2,) * 8 + (67,), "identity"), ((7, 2, 4), "identity"), ((7, 2, 4), "random")])
 def test_split_kernel_reports_unsupported(radices, perm):
     spec = wl.make_plan(3, int(np.prod(radices)), radices, "qr", perm=perm)
     plan = harp.plan_from_spec(spec)
