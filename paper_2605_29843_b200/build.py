@@ -38,6 +38,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         cmd += ["-DHARP_TM_TIMING"]
     if os.environ.get("HARP_FAST_TIMING"):        # ... and in the whole-row kernel
         cmd += ["-DHARP_FAST_TIMING"]
+    if os.environ.get("HARP_UPPER_TIMING"):       # ... and in the dense upper pass (printed by CTA 0)
+        cmd += ["-DHARP_UPPER_TIMING"]
     cmd += sources() + ["-o", LIB]
     subprocess.check_call(cmd)
     return LIB

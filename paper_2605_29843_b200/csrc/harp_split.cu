@@ -28,6 +28,7 @@
 // before the passes in the forward direction, after them in the transpose direction.  The sign
 // diagonal stays folded into the first phase's fragments, read through the permutation.
 #include <algorithm>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -315,6 +316,7 @@ harp_split_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_
 // by the copies (eight 16-byte loads -> 8x8 transpose -> eight 16-byte stores).
 struct UpperPass {
     int32_t n_cg, Lw, U, KP, NT, pitch, MT;
+    int32_t l_skew;            // elements added to the tile offset of a position per octet of positions
     int32_t S_mid, row_stride;
     const uint32_t *bfrag;     // [column group][l][n-tile][k-step][lane][2]
     int32_t bfrag_words;
@@ -422,6 +424,162 @@ harp_upper_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_
     cp_async_wait_all();
 }
 
+// The same pass with the fragments of F_l in registers (KS <= 3, i.e. U <= 48): warp w owns positions
+// w and w + 8 of a column group of sixteen, loads their fragments once from global memory and keeps
+// them for every row the CTA sees.  Shared memory holds the tile twice: a staging buffer that cp.async
+// fills with the rows as they are in global memory ([row][octet of l][u][8 values of l], the 16-byte
+// chunks of a u-octet XOR-swizzled by the octet's index), and the operand buffer [row][l][u] that the
+// transposing copy (eight 16-byte loads -> 8x8 transpose in registers -> eight 16-byte stores) writes
+// and ldmatrix / stmatrix work on.  The staging buffer of the next tile fills while this tile is
+// multiplied and written back, so the copy's latency is hidden without holding registers for it.
+// The positions of the second octet are shifted by l_skew elements in the operand buffer so that the
+// two position octets of a transposing copy fall into different bank groups.
+// Per-section cycle counts of harp_upper_reg_kernel (build with -DHARP_UPPER_TIMING): thread 0 of CTA 0 prints
+// the cycles it spent in  0 wait for the staged rows | 1 transposing copy | 2 issue of the next stage |
+// 3 products | 4 copy out.
+#ifdef HARP_UPPER_TIMING
+#define UP_DECL long long up_acc[5] = {0, 0, 0, 0, 0}, up_last = clock64()
+#define UP_MARK(k) do { if (threadIdx.x == 0) { const long long now_ = clock64(); up_acc[k] += now_ - up_last; up_last = now_; } } while (0)
+#define UP_DUMP do { if (threadIdx.x == 0 && blockIdx.x == 0) printf("upper sections: wait %lld  transpose %lld  stage %lld  products %lld  out %lld  tiles %lld\n", up_acc[0], up_acc[1], up_acc[2], up_acc[3], up_acc[4], (long long)((n_tiles - part + n_parts - 1) / n_parts)); } while (0)
+#else
+#define UP_DECL do { } while (0)
+#define UP_MARK(k) do { } while (0)
+#define UP_DUMP do { } while (0)
+#endif
+
+template <int KS>
+__global__ void __launch_bounds__(kSplitThreads, 2)
+harp_upper_reg_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_end, UpperPass P) {
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int pitch = P.pitch, MT = P.MT, KP = P.KP, NT = P.NT, U = P.U;
+    const int tile_rows = 16 * MT;
+    const uint32_t sbase = smem_u32(smem_raw);                                  // operand buffer
+    const uint32_t stage = sbase + (uint32_t)(((size_t)tile_rows * pitch * 2 + 15) / 16 * 16);
+    const uint32_t stage_row = 32u * (uint32_t)KP + 64u;                        // bytes per row: 2 octets of l x KP chunks, the second shifted by 4 chunks
+    const int cg = blockIdx.x % P.n_cg, part = blockIdx.x / P.n_cg, n_parts = gridDim.x / P.n_cg;
+    __nv_bfloat16 *xg = x + (size_t)cg * P.Lw;
+    const int64_t n_tiles = (row_end - row_begin + tile_rows - 1) / tile_rows;
+    const int64_t rs = P.row_stride;
+    // fragments of this warp's two positions
+    uint2 bfr[2][2 * KS][KS];
+#pragma unroll
+    for (int li = 0; li < 2; ++li) {
+        const uint2 *src = reinterpret_cast<const uint2 *>(P.bfrag + (size_t)cg * P.bfrag_words) +
+                           (size_t)(warp + 8 * li) * NT * KS * 32 + lane;
+#pragma unroll
+        for (int nt = 0; nt < 2 * KS; ++nt)
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks)
+                bfr[li][nt][ks] = nt < NT ? __ldg(src + (nt * KS + ks) * 32) : make_uint2(0u, 0u);
+    }
+    // transposing copies: a thread owns one (octet of l, octet of u) unit and walks over rows
+    const int uo_n = KP >> 3;
+    const int units_per_row = 2 * uo_n;
+    const int cp_rows = kSplitThreads / units_per_row;
+    const int cp_r = threadIdx.x / units_per_row, un = threadIdx.x - cp_r * units_per_row;
+    const int lo = un / uo_n, uo = un - lo * uo_n;
+    const int unit_off = (8 * lo) * KP + lo * P.l_skew + 8 * uo;
+    const uint32_t unit_stage = (uint32_t)(lo * (KP + 4) + 8 * uo) * 16u;
+    // copy out: the two position octets of a (row, u) in neighbouring lanes, so that a pair of lanes writes a whole sector
+    const int lo_w = un & 1, uo_w = un >> 1;
+    const int unit_off_w = (8 * lo_w) * KP + lo_w * P.l_skew + 8 * uo_w;
+
+    // rows of a tile as they are, into the staging buffer: chunk = (row, u, octet of l); a thread's chunks are
+    // kSplitThreads apart in (row, u, l8) order, stepped without a division
+    const int per_row = 2 * U;
+    const int c_r0 = threadIdx.x / per_row, c_rem0 = threadIdx.x - c_r0 * per_row;
+    const int step_r = kSplitThreads / per_row, step_rem = kSplitThreads - step_r * per_row;
+    auto stage_in = [&](int64_t tile) {
+        const int64_t row0 = row_begin + tile * tile_rows;
+        int r = c_r0, rem = c_rem0;
+        while (r < tile_rows) {
+            const int u = rem >> 1, l8 = rem & 1;
+            const int64_t row = min(row0 + r, row_end - 1);
+            const uint32_t dst = stage + (uint32_t)r * stage_row + (uint32_t)(l8 * (KP + 4) + (u & ~7) + ((u & 7) ^ ((u >> 3) & 7))) * 16u;
+            cp_async16(dst, xg + row * rs + (int64_t)u * P.S_mid + 8 * l8);
+            r += step_r;
+            rem += step_rem;
+            if (rem >= per_row) { rem -= per_row; ++r; }
+        }
+        cp_async_commit();
+    };
+
+    rows_ready_barrier();
+    UP_DECL;
+    if (part < n_tiles) stage_in(part);
+    for (int64_t tile = part; tile < n_tiles; tile += n_parts) {
+        const int64_t row0 = row_begin + tile * tile_rows;
+        cp_async_wait_group<0>();
+        __syncthreads();
+        UP_MARK(0);
+        // ---- staging buffer -> operand buffer, transposing: unit = (row, octet of l, octet of u)
+        for (int r = cp_r; r < tile_rows && cp_r < cp_rows; r += cp_rows) {
+            const uint32_t src = stage + (uint32_t)r * stage_row + unit_stage;
+            uint4 in[8], out[8];
+#pragma unroll
+            for (int uu = 0; uu < 8; ++uu)
+                in[uu] = 8 * uo + uu < U ? lds128(src + 16u * (uint32_t)(uu ^ (uo & 7))) : make_uint4(0u, 0u, 0u, 0u);
+            transpose8x8_b16(in, out);
+            const uint32_t dst = sbase + 2u * (uint32_t)(r * pitch + unit_off);
+#pragma unroll
+            for (int ll = 0; ll < 8; ++ll) sts128(dst + 2u * (uint32_t)(ll * KP), out[ll]);
+        }
+        __syncthreads();
+        UP_MARK(1);
+        if (tile + n_parts < n_tiles) stage_in(tile + n_parts);       // lands under the products and the copy out
+        UP_MARK(2);
+
+        // ---- one dense block per (l, row group); the fragments stay where they are
+        {
+            const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
+#pragma unroll
+            for (int li = 0; li < 2; ++li) {
+                const uint32_t addr0 = sbase + 2u * (uint32_t)(mrow * pitch + (warp + 8 * li) * KP + li * P.l_skew + mcol);
+                for (int mt = 0; mt < MT; ++mt) {
+                    const uint32_t addr = addr0 + 32u * (uint32_t)(mt * pitch);
+                    uint32_t a[KS][4];
+#pragma unroll
+                    for (int ks = 0; ks < KS; ++ks) ldmatrix_x4(a[ks], addr + 32u * ks);
+#pragma unroll
+                    for (int c = 0; c < KS; ++c) {
+                        float acc[2][4];
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            acc[h][0] = acc[h][1] = acc[h][2] = acc[h][3] = 0.f;
+#pragma unroll
+                            for (int ks = 0; ks < KS; ++ks) mma_k16_acc(acc[h], a[ks], bfr[li][2 * c + h][ks].x, bfr[li][2 * c + h][ks].y);
+                        }
+                        stmatrix_x4(addr + 32u * c, pack_bf16(acc[0][0], acc[0][1]), pack_bf16(acc[0][2], acc[0][3]),
+                                    pack_bf16(acc[1][0], acc[1][1]), pack_bf16(acc[1][2], acc[1][3]));
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        UP_MARK(3);
+
+        // ---- copy out, transposing back
+        for (int r = cp_r; r < tile_rows && cp_r < cp_rows && row0 + r < row_end; r += cp_rows) {
+            const uint32_t srcs = sbase + 2u * (uint32_t)(r * pitch + unit_off_w);
+            uint4 in[8], out[8];
+#pragma unroll
+            for (int ll = 0; ll < 8; ++ll) in[ll] = lds128(srcs + 2u * (uint32_t)(ll * KP));
+            transpose8x8_b16(in, out);
+            __nv_bfloat16 *dstg = xg + (row0 + r) * rs + 8 * lo_w;
+#pragma unroll
+            for (int uu = 0; uu < 8; ++uu) {
+                const int u = 8 * uo_w + uu;
+                if (u < U) stg128(dstg + (int64_t)u * P.S_mid, out[uu]);
+            }
+        }
+        // (the next iteration's barrier separates these reads from the next transposing copy)
+        UP_MARK(4);
+    }
+    UP_DUMP;
+    cp_async_wait_all();
+}
+
 // ---------------------------------------------------------------------------------------
 // Fixed permutation of wide rows, in place: out[i] = in[table[i]] for every row (Theorem 1's
 // permutation convention: table = the plan's permutation in the forward direction, its inverse
@@ -503,6 +661,7 @@ struct SplitPlan {
     size_t gather_smem = 0;
     // dense upper pass (replaces pass[1] when set)
     bool dense_upper = false;
+    bool up_in_regs = false;   // fragments in registers (harp_upper_reg_kernel)
     UpperPass up_fwd{}, up_bwd{};
     size_t up_smem = 0;
     int up_ks = 0;
@@ -733,15 +892,21 @@ harp_status_t build_dense_upper(const harp_plan *plan, SplitPlan *sp, int t0, in
     if (U > 64 || U < 2) return HARP_ERR_UNSUPPORTED;
     const int KP = (int)((U + 15) / 16 * 16), KS = KP / 16, NT = (int)((U + 7) / 8);
     const int64_t per_l_words = (int64_t)NT * KS * 64;
+    // U <= 48 and sixteen positions per column group: the fragments of two positions fit a warp's registers
+    const bool in_regs = KS <= 3 && S_mid % 16 == 0;
     int Lw = 16;
-    if (S_mid % 16 != 0 || 16 * per_l_words * 4 > 80 * 1024) Lw = 8;
+    if (!in_regs && (S_mid % 16 != 0 || 16 * per_l_words * 4 > 80 * 1024)) Lw = 8;
     if (S_mid % Lw != 0) return HARP_ERR_UNSUPPORTED;
-    int64_t pitch = (int64_t)Lw * KP;
+    const int l_skew = in_regs ? 32 : 0;
+    int64_t pitch = (int64_t)Lw * KP + l_skew;
     if ((pitch / 8) % 2 == 0) pitch += 8;
-    const int64_t frag_bytes = Lw * per_l_words * 4;
+    const int64_t frag_bytes = in_regs ? 0 : Lw * per_l_words * 4;
     int MT = 1;
-    while (MT < 4 && (int64_t)32 * MT * pitch * 2 + frag_bytes <= 100 * 1024) MT *= 2;
-    const size_t smem = ((size_t)16 * MT * pitch * 2 + 15) / 16 * 16 + (size_t)frag_bytes;
+    // in_regs: the tile twice (operand buffer and the staging buffer of 32 KP + 64 bytes per row)
+    auto tile_bytes = [&](int mt) { return (int64_t)16 * mt * (pitch * 2 + (in_regs ? 32 * KP + 64 : 0)); };
+    while (MT < 4 && tile_bytes(2 * MT) + frag_bytes <= (in_regs ? 110 : 100) * 1024) MT *= 2;
+    const size_t smem = in_regs ? ((size_t)16 * MT * pitch * 2 + 15) / 16 * 16 + (size_t)16 * MT * (32 * KP + 64)
+                                : ((size_t)16 * MT * pitch * 2 + 15) / 16 * 16 + (size_t)frag_bytes;
     if (smem > 110u * 1024u) return HARP_ERR_UNSUPPORTED;
     if ((Lw / 8) * (KP / 8) > kSplitThreads) return HARP_ERR_UNSUPPORTED;
     const int n_cg = (int)(S_mid / Lw);
@@ -751,6 +916,7 @@ harp_status_t build_dense_upper(const harp_plan *plan, SplitPlan *sp, int t0, in
     for (int dir = 0; dir < 2 && st == HARP_OK; ++dir) {
         UpperPass &P = dir == 0 ? sp->up_fwd : sp->up_bwd;
         P.n_cg = n_cg; P.Lw = Lw; P.U = (int32_t)U; P.KP = KP; P.NT = NT; P.pitch = (int32_t)pitch; P.MT = MT;
+        P.l_skew = l_skew;
         P.S_mid = (int32_t)S_mid; P.row_stride = (int32_t)plan->d;
         P.bfrag_words = (int32_t)(Lw * per_l_words);
         std::vector<uint32_t> frag((size_t)n_cg * P.bfrag_words, 0u);
@@ -776,6 +942,7 @@ harp_status_t build_dense_upper(const harp_plan *plan, SplitPlan *sp, int t0, in
         P.bfrag = upload_s(sp, frag, st);
     }
     sp->dense_upper = true;
+    sp->up_in_regs = in_regs;
     sp->up_smem = smem;
     sp->up_ks = KS;
     return st;
@@ -828,7 +995,10 @@ harp_status_t harp_split_build(harp_plan *plan) {
          cudaFuncSetAttribute(harp_upper_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess ||
          cudaFuncSetAttribute(harp_upper_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess ||
          cudaFuncSetAttribute(harp_upper_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess ||
-         cudaFuncSetAttribute(harp_upper_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess))
+         cudaFuncSetAttribute(harp_upper_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess ||
+         cudaFuncSetAttribute(harp_upper_reg_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess ||
+         cudaFuncSetAttribute(harp_upper_reg_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess ||
+         cudaFuncSetAttribute(harp_upper_reg_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 110 * 1024) != cudaSuccess))
         st = HARP_ERR_CUDA;
     if (st == HARP_OK && permuted) {
         std::vector<uint16_t> fwd((size_t)d), bwd((size_t)d);
@@ -931,6 +1101,13 @@ harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, h
                 parts = std::min(parts, n_tiles);
                 const unsigned grid = (unsigned)(parts * P.n_cg);
                 cudaError_t err;
+                if (sp->up_in_regs) {
+                    switch (sp->up_ks) {
+                        case 1: err = launch_pass(harp_upper_reg_kernel<1>, grid, sp->up_smem, stream, overlap, xb, r0, r1, P); break;
+                        case 2: err = launch_pass(harp_upper_reg_kernel<2>, grid, sp->up_smem, stream, overlap, xb, r0, r1, P); break;
+                        default: err = launch_pass(harp_upper_reg_kernel<3>, grid, sp->up_smem, stream, overlap, xb, r0, r1, P); break;
+                    }
+                } else
                 switch (sp->up_ks) {
                     case 1: err = launch_pass(harp_upper_kernel<1>, grid, sp->up_smem, stream, overlap, xb, r0, r1, P); break;
                     case 2: err = launch_pass(harp_upper_kernel<2>, grid, sp->up_smem, stream, overlap, xb, r0, r1, P); break;
