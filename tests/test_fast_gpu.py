@@ -38,6 +38,29 @@ def test_fast_kernel_matches_oracle(radices, perm, kind):
                 assert orc.rel_err_rows(got, want) <= TOL["bf16"]
 
 
+@pytest.mark.parametrize("radices,perm", [((4,) * 6, "digit_reversal"), ((4,) * 6, "identity"), ((16, 16, 8), "digit_reversal")])
+def test_several_tiles_per_cta_and_a_ragged_last_tile(radices, perm):
+    """More tiles than SMs, so that a CTA works through several tiles, and row counts that leave the last tile
+    partly empty.  For the largest count a sample of rows (both ends of the batch and rows in between) is
+    compared, otherwise every row."""
+    spec = wl.make_plan(29, int(np.prod(radices)), radices, "qr", perm=perm, signs=True)
+    oplan = orc.OraclePlan.from_spec(spec)
+    plan = harp.plan_from_spec(spec)
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    rng = np.random.default_rng(12)
+    for n_rows in (16 * sms * 2 + 7, 16 * sms + 16 * 3 + 1, 12 * sms * 6 + 12 * 5 + 5):
+        xh = host_rows(rng.standard_normal((n_rows, spec.d)), "bf16")
+        pick = np.arange(n_rows)
+        if n_rows > 6000:
+            pick = np.unique(np.concatenate([np.arange(40), np.arange(n_rows - 40, n_rows), rng.integers(0, n_rows, 300)]))
+        x64 = promote(xh[pick], "bf16")
+        for tr in (False, True):
+            got, guards = gpu_apply(plan, xh, "bf16", tr, harp.KERNEL_FAST)
+            want = orc.transpose(oplan, x64) if tr else orc.forward(oplan, x64)
+            assert guards
+            assert orc.rel_err_rows(got[pick], want) <= TOL["bf16"]
+
+
 @pytest.mark.parametrize("radices,perm,dtype", [((16, 16, 8, 7), "identity", "bf16"), ((4,) * 6, "random", "bf16"),
                                                 ((4,) * 6, "identity", "f32"), ((2,) * 9, "identity", "bf16")])
 def test_fast_kernel_reports_unsupported(radices, perm, dtype):
