@@ -23,18 +23,25 @@ import numpy as np
 
 
 def greedy_schedule(d: int, b_base: int = 8, b_max: int = 8) -> List[int]:
+    """Algorithm 2 as a recurrence on the part of d not yet factored: the next stage takes the preferred
+    radix b_base while it divides what is left, otherwise the largest divisor of what is left that does
+    not exceed b_max, and a remainder without such a divisor becomes the last stage itself."""
     if d < 2:
         raise ValueError("d >= 2 required")
-    out, r = [], d
-    while r % b_base == 0:                       # peel the preferred radix
-        out.append(b_base)
-        r //= b_base
-    for f in range(min(b_max, r), 1, -1):        # largest admissible factors first
-        while r % f == 0:
-            out.append(f)
-            r //= f
-    if r != 1:                                   # leftover factor as a final stage
-        out.append(r)
+
+    def next_radix(rest: int, base_allowed: bool):
+        if base_allowed and rest % b_base == 0:
+            return b_base, True
+        for f in range(min(b_max, rest), 1, -1):
+            if rest % f == 0:
+                return f, False
+        return rest, False
+
+    out, rest, base_allowed = [], d, True
+    while rest > 1:
+        b, base_allowed = next_radix(rest, base_allowed)
+        out.append(b)
+        rest //= b
     return out
 
 
