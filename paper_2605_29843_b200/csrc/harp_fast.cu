@@ -224,6 +224,12 @@ harp_fast_kernel(__nv_bfloat16 *__restrict__ x, int64_t n_rows, int64_t n_tiles,
         const long long wait = (long long)(blockIdx.x % 3) * stagger, t0 = clock64();
         while (clock64() - t0 < wait) { }
     }
+    // Everything above reads the plan's data only.  Launched with the programmatic stream-serialisation
+    // attribute, a CTA gets here while the kernel before it in the stream is still running on other SMs
+    // (tables, tensor-memory fill and the start delay then cost nothing); the rows are touched only after
+    // that kernel has completed.  The kernel after this one may start its own preamble as SMs become free.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 #ifdef HARP_FAST_TIMING
     long long tacc[16] = {0}, tlast = clock64();
 #endif
@@ -1049,10 +1055,21 @@ harp_status_t harp_fast_apply(const harp_plan *plan, void *x, int64_t n_rows, ha
     // a quarter of a tile period, estimated from the measured 28 k cycles per tile of d = 4096 with
     // three phases (the gain is flat between half and the full value)
     const int stagger = n_tiles >= 4 * (int64_t)grid ? (int)(0.57 * (double)P.d * P.n_phases) : 0;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = fp->smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t err;
     switch (transpose ? fp->variant_bwd : fp->variant_fwd) {
-        case 1: harp_fast_kernel<kThreads, kModesReorderOut><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, stagger, P); break;
-        default: harp_fast_kernel<kThreads, kModesGeneral><<<grid, kThreads, fp->smem_bytes, stream>>>(xb, n_rows, n_tiles, stagger, P); break;
+        case 1: err = cudaLaunchKernelEx(&cfg, harp_fast_kernel<kThreads, kModesReorderOut>, xb, n_rows, n_tiles, stagger, P); break;
+        default: err = cudaLaunchKernelEx(&cfg, harp_fast_kernel<kThreads, kModesGeneral>, xb, n_rows, n_tiles, stagger, P); break;
     }
     g_harp_launches.fetch_add(1, std::memory_order_relaxed);
-    return cudaGetLastError() == cudaSuccess ? HARP_OK : HARP_ERR_CUDA;
+    return err == cudaSuccess && cudaGetLastError() == cudaSuccess ? HARP_OK : HARP_ERR_CUDA;
 }
