@@ -172,6 +172,11 @@ harp_tm_kernel(const __grid_constant__ CUtensorMap tmap, const TmParams P) {
     tc_fence_after();
     const uint32_t tmem = tmem_base_s;
     const Waiter wait{&dead_s, P.err};
+    // Barriers and tensor memory are set up; nothing above touches the rows.  Launched with the programmatic
+    // stream-serialisation attribute this point is reached while the kernel before this one in the stream is
+    // still finishing on other SMs; the rows are read and written only after it has completed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     const int64_t n_tiles = (int64_t)P.n_row_tiles * P.n_col_tiles;
     const int64_t t_begin = (int64_t)blockIdx.x * P.tiles_per_cta;
@@ -578,8 +583,18 @@ cudaError_t launch_one(const CUtensorMap &map, const TmParams &prm, int grid, si
         attr = cudaFuncSetAttribute(harp_tm_kernel<FMT, K0, K1, XP>, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448 - 1024);
     });
     if (attr != cudaSuccess) return attr;
-    harp_tm_kernel<FMT, K0, K1, XP><<<grid, kThreads, smem, s>>>(map, prm);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute la[1];
+    la[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    la[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = la;
+    cfg.numAttrs = 1;
+    const cudaError_t err = cudaLaunchKernelEx(&cfg, harp_tm_kernel<FMT, K0, K1, XP>, map, prm);
+    return err != cudaSuccess ? err : cudaGetLastError();
 }
 
 }  // namespace
