@@ -259,11 +259,15 @@ harp_split_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_
                     const int it = w >> mt_shift, mt = w & (MT - 1);
                     const uint32_t a0 = sbase + 2u * (uint32_t)((mt * 16 + g) * pitch + tab_s[ph.items_off + it]);
                     const uint32_t a1 = a0 + 16u * (uint32_t)pitch;
-                    const uint32_t bfa = bf_s + 4u * (uint32_t)(ph.bfrag_off + it * 256 + lane);
+                    // the eight blocks' fragment words of a lane: two 16-byte loads ([half][lane][4 words] per item)
+                    const uint32_t bfa = bf_s + 4u * (uint32_t)(ph.bfrag_off + it * 256 + lane * 4);
                     uint4 raw[2][2];
                     uint32_t bf[8];
-#pragma unroll
-                    for (int e = 0; e < 8; ++e) bf[e] = lds32(bfa + e * 128);
+                    {
+                        const uint4 f0 = lds128(bfa), f1 = lds128(bfa + 512);
+                        bf[0] = f0.x; bf[1] = f0.y; bf[2] = f0.z; bf[3] = f0.w;
+                        bf[4] = f1.x; bf[5] = f1.y; bf[6] = f1.z; bf[7] = f1.w;
+                    }
 #pragma unroll
                     for (int j = 0; j < 2; ++j) {
                         raw[j][0] = lds128(a0 + so[j]);
@@ -854,9 +858,13 @@ harp_status_t build_pass(const harp_plan *plan, SplitPlan *sp, PassHost &ph_out,
                     };
                     auto slot = [&](int s) { return is.mode == 0 ? s : strided_slot(s, B, l); };
                     uint32_t *dst0 = frag.data() + (size_t)cgi * words + frag_off[(size_t)p] + bi * 32 * wpl;
+                    // 8-wide strided phases: the words of an item's eight blocks sit together per lane,
+                    // [item][blocks 0-3 | 4-7][lane][4 words], so that a lane fetches them with two 16-byte loads
+                    const bool grouped = is.mode == 1 && B == 8;
+                    uint32_t *grp0 = frag.data() + (size_t)cgi * words + frag_off[(size_t)p] + (bi / 8) * 256 + ((bi % 8) / 4) * 128 + (bi % 4);
                     for (int lane = 0; lane < 32; ++lane) {
                         const int gg = lane >> 2, qq = lane & 3;
-                        uint32_t *dst = dst0 + lane * wpl;
+                        uint32_t *dst = grouped ? grp0 + lane * 4 : dst0 + lane * wpl;
                         if (B == 16) {
                             for (int nt = 0; nt < 2; ++nt) {
                                 const int n = slot(8 * nt + gg);
