@@ -53,6 +53,7 @@ struct SplitPhase {
     int32_t lm, jr[4];         // local index of slot j of lane q is lm*q + jr[j]
     int32_t items_off, n_items;
     int32_t bfrag_off;         // word offset of the phase's fragments inside a column group's block
+    int32_t paired;            // mode 0, B = 8: blocks 2k and 2k+1 are neighbours in the tile; a warp takes both at once
 };
 
 struct SplitPass {
@@ -194,6 +195,25 @@ harp_split_kernel(__nv_bfloat16 *__restrict__ x, int64_t row_begin, int64_t row_
                             float c0[4], c1[4];
                             mma_k16(c0, a, bf.x, bf.y);
                             mma_k16(c1, a, bf.z, bf.w);
+                            stmatrix_x4(addr, pack_bf16(c0[0], c0[1]), pack_bf16(c0[2], c0[3]), pack_bf16(c1[0], c1[1]),
+                                        pack_bf16(c1[2], c1[3]));
+                        }
+                    }
+                } else if (ph.paired) {
+                    // two neighbouring 8-wide blocks per ldmatrix.x4 / stmatrix.x4: half the shared-memory instructions
+                    const int mrow = (lane & 7) + ((lane >> 3) & 1) * 8, mcol = (lane >> 4) * 8;
+                    const uint32_t lane_addr = sbase + 2u * (uint32_t)(mrow * pitch + mcol);
+                    for (int it = 2 * warp; it < ph.n_items; it += 2 * kSplitWarps) {
+                        const uint32_t bfa = bf_s + 4u * (uint32_t)(ph.bfrag_off + it * 32 + lane);
+                        const uint32_t bf0 = lds32(bfa), bf1 = lds32(bfa + 128);
+                        uint32_t addr = lane_addr + 2u * (uint32_t)tab_s[ph.items_off + it];
+                        for (int mt = 0; mt < MT; ++mt, addr += 32u * (uint32_t)pitch) {
+                            uint32_t a[4];
+                            ldmatrix_x4(a, addr);
+                            const uint32_t a_lo[2] = {a[0], a[1]}, a_hi[2] = {a[2], a[3]};
+                            float c0[4], c1[4];
+                            mma_k8(c0, a_lo, bf0);
+                            mma_k8(c1, a_hi, bf1);
                             stmatrix_x4(addr, pack_bf16(c0[0], c0[1]), pack_bf16(c0[2], c0[3]), pack_bf16(c1[0], c1[1]),
                                         pack_bf16(c1[2], c1[3]));
                         }
@@ -809,6 +829,11 @@ harp_status_t build_pass(const harp_plan *plan, SplitPlan *sp, PassHost &ph_out,
             for (int j = 0; j < 4; ++j) { D.jr[j] = jo[j]; D.j_off[j] = (int32_t)(jo[j] * W[(size_t)p]); }
             D.items_off = (int32_t)tab.size();
             D.n_items = (int32_t)is.bases.size();
+            D.paired = 0;
+            if (is.mode == 0 && gp.B == 8 && is.bases.size() % 2 == 0) {
+                D.paired = 1;
+                for (size_t i = 0; i + 1 < is.bases.size(); i += 2) D.paired = D.paired && is.bases[i + 1] == is.bases[i] + 8;
+            }
             tab.insert(tab.end(), is.bases.begin(), is.bases.end());
             D.bfrag_off = words;
             frag_off[(size_t)p] = words;
