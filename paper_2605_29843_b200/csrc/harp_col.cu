@@ -127,6 +127,29 @@ harp_col_kernel(__nv_bfloat16 *__restrict__ W, int64_t ld, int64_t n_cols, ColPa
                                       pack_bf16(c1f[2], c1f[3]));
                     }
                 }
+            } else if ((MT & 1) == 0) {
+                // 8-wide blocks: two 16-column groups per ldmatrix.x4 / stmatrix.x4 (lanes 16-31 address the second
+                // group), the block's fragment used twice: half the shared-memory instructions
+                const int k = lane & 7, mch = lane >> 3;
+                const bool real = k < ph.B_real;
+                const uint32_t lane_ld = sbase + (uint32_t)((real ? k * ph.wr : 0) * rowbytes + 16 * mch);
+                const uint32_t lane_scr = sbase + (uint32_t)(scratch_row * rowbytes + 16 * mch);
+                for (int it = warp; it < ph.n_items; it += kColWarps) {
+                    const uint32_t row_off = (uint32_t)(tab_s[ph.items_off + it] * rowbytes);
+                    const uint32_t bf = lds32c(bf_s + 4u * (uint32_t)(ph.bfrag_off + it * 32 + lane));
+                    uint32_t ld_addr = lane_ld + row_off, st_addr = real ? ld_addr : lane_scr;
+#pragma unroll 2
+                    for (int mt = 0; mt < MT; mt += 2, ld_addr += 64, st_addr += 64) {
+                        uint32_t a[4];
+                        ldmatrix_x4_t(a, ld_addr);
+                        const uint32_t a_lo[2] = {a[0], a[1]}, a_hi[2] = {a[2], a[3]};
+                        float c0f[4], c1f[4];
+                        mma_k8(c0f, a_lo, bf);
+                        mma_k8(c1f, a_hi, bf);
+                        stmatrix_x4_t(st_addr, pack_bf16(c0f[0], c0f[1]), pack_bf16(c0f[2], c0f[3]), pack_bf16(c1f[0], c1f[1]),
+                                      pack_bf16(c1f[2], c1f[3]));
+                    }
+                }
             } else {
                 const int k = lane & 7, mch = (lane >> 3) & 1;
                 const bool real = k < ph.B_real;
