@@ -147,3 +147,42 @@ def test_small_batches_chained_and_in_a_cuda_graph(n_rows):
     # five roundings to bf16 along the chain: a few times the single-apply tolerance
     want = orc.forward(oplan, promote(xh, "bf16"))
     assert orc.rel_err_rows(to_host_f64(eager), want) <= 3 * TOL["bf16"]
+
+
+@pytest.mark.parametrize("cfg,n_rows", [(2, 48), (2, 16 * 300 + 5), (4, 2048)])
+def test_dependent_launches_chained_and_in_a_cuda_graph(cfg, n_rows):
+    """The whole-row kernel (cfg2) and the tensor-memory slab pass (cfg4 from 1024 rows on) start their
+    preamble while the kernel before them in the stream is still running and touch the rows only after it has
+    completed.  A forward/transpose chain on a side stream must give the same bits whether launched call by
+    call or replayed from a CUDA graph, and match the oracle on a sample of rows."""
+    spec = wl.config(cfg).plans["q"]
+    plan = harp.plan_from_spec(spec)
+    oplan = orc.OraclePlan.from_spec(spec)
+    rng = np.random.default_rng(190 + n_rows)
+    xh = host_rows(rng.standard_normal((n_rows, spec.d)), "bf16")
+    side = torch.cuda.Stream()
+
+    def chain(x, st):
+        for k in range(5):                                  # F T F T F: one forward in total
+            harp.harp_apply(plan, x.data_ptr(), n_rows, harp.HARP_BF16, bool(k & 1), st)
+
+    eager = to_device(xh, "bf16")
+    with torch.cuda.stream(side):
+        chain(eager, side.cuda_stream)
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    scratch = to_device(xh, "bf16")
+    fresh = to_device(xh, "bf16")
+    with torch.cuda.stream(side):
+        chain(scratch, side.cuda_stream)                    # warm-up before capture
+        side.synchronize()
+        scratch.copy_(fresh)
+        with torch.cuda.graph(graph, stream=side):
+            chain(scratch, side.cuda_stream)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(eager.view(torch.int16), scratch.view(torch.int16))
+    pick = np.unique(np.concatenate([np.arange(min(n_rows, 24)), np.arange(max(0, n_rows - 24), n_rows)]))
+    want = orc.forward(oplan, promote(xh[pick], "bf16"))
+    assert orc.rel_err_rows(to_host_f64(eager)[pick], want) <= 3 * TOL["bf16"]
+    assert harp.harp_plan_error_word(plan) == 0
