@@ -161,7 +161,10 @@ int64_t harp_plan_dim(const harp_plan_t *plan);
  *   x        DEVICE n_rows x d, dtype fp32 or bf16, overwritten with the result
  *   stream   a cudaStream_t passed as void* (NULL = default stream)
  * Asynchronous on stream; does not synchronise.  n_rows == 0 returns HARP_OK without
- * a launch.  A plan may be applied from several streams at once.
+ * a launch.  A plan may be applied from several streams at once.  Stream order holds as for
+ * any kernel; some kernels are launched so that their set-up (plan data only) may begin while
+ * earlier work in the stream is still running -- they read and write x only after that work
+ * has completed.
  * Arithmetic.  fp32 rows: fp32 block kernels, fp32 accumulate, the result is the fp32 sum (one
  * rounding per stage).  bf16 rows on the tensor-core kernels (what HARP_KERNEL_AUTO picks for
  * bf16 whenever a plan has one): neighbouring stages are fused at plan time into dense blocks of
