@@ -748,7 +748,10 @@ harp_status_t build_pass(const harp_plan *plan, SplitPlan *sp, PassHost &ph_out,
     const int n_cg = lower ? (int)U : (int)(S_mid / inner);
     const int n_chunks = lower ? (int)(S_mid / 8) : (int)(U * inner / 8);
     // rows per tile: as many 16-row groups as fit ~40 KB
-    int MT = (int)std::max<int64_t>(1, std::min<int64_t>(4, (40 * 1024) / (pitch * 2 * 16)));
+    // (measured on 65536 rows of d = 28672: slabs of 512 coordinates with 64-row tiles and two CTAs per SM are 4 %
+    // faster than with 32-row tiles and three; for the position groups of the upper pass larger tiles gain nothing.
+    // The launch shrinks the tile for batches that do not fill it.)
+    int MT = (int)std::max<int64_t>(1, std::min<int64_t>(4, ((lower ? 80 : 40) * 1024) / (pitch * 2 * 16)));
     if (MT == 3) MT = 2;
     if (n_chunks > 4 * kSplitThreads) return HARP_ERR_UNSUPPORTED;
 
@@ -1161,7 +1164,11 @@ harp_status_t harp_split_apply(const harp_plan *plan, void *x, int64_t n_rows, h
                 if (ts != HARP_ERR_UNSUPPORTED) return ts;
             }
             const PassHost &ph = sp->pass[pi];
-            const SplitPass &P = transpose ? ph.bwd : ph.fwd;
+            SplitPass P = transpose ? ph.bwd : ph.fwd;
+            while (P.MT > 1 && 16 * (int64_t)(P.MT / 2) >= r1 - r0) {     // a small batch takes the smallest tile that holds it
+                P.MT /= 2;
+                --P.mt_shift;
+            }
             const int64_t tile_rows = 16 * P.MT;
             const int64_t n_tiles = (r1 - r0 + tile_rows - 1) / tile_rows;
             // one wave of CTAs, each keeping its column group for as many tiles as possible
