@@ -401,7 +401,9 @@ harp_status_t harp_col_apply(const harp_plan *plan, void *W, int64_t n_cols, int
     for (int s = 0; s < cp->n_pass; ++s) {
         const ColPass &P = cp->pass[s];
         const int64_t n_tiles = (n_cols + P.NC - 1) / P.NC;
-        const int per_sm = std::max<int>(1, std::min<int>(2, (int)((220 * 1024) / (cp->smem[s] + 1024))));
+        // up to three CTAs per SM (70 registers per thread): the pass with the small tile gains from the third
+        // (two-sided product of the 8192 x 28672 matrix 1.14 -> 1.10 ms); 32-column tiles were measured slower
+        const int per_sm = std::max<int>(1, std::min<int>(3, (int)((220 * 1024) / (cp->smem[s] + 1024))));
         int64_t parts = std::max<int64_t>(1, ((int64_t)cp->sms * per_sm) / P.n_cg);
         parts = std::min(parts, n_tiles);
         harp_col_kernel<<<(unsigned)(parts * P.n_cg), kColThreads, cp->smem[s], stream>>>(static_cast<__nv_bfloat16 *>(W), ld, n_cols, P);
