@@ -86,7 +86,7 @@ def test_split_kernel_matches_oracle(radices, kind):
     plan = harp.plan_from_spec(spec)
     rng = np.random.default_rng(9)
     big = 2100 if spec.d > 10000 else 600            # more rows than one L2 chunk for the wide plans
-    for n_rows in (1, 16, 37, big):
+    for n_rows in (1, 16, 17, 33, 37, big):          # 17 and 33: just past the 16- and 32-row tiles a small batch takes
         xh = host_rows(rng.standard_normal((n_rows, spec.d)), "bf16")
         x64 = promote(xh, "bf16")
         for tr in (False, True):
