@@ -31,6 +31,7 @@
 // permutations use the generic kernel.
 #include <algorithm>
 #include <cmath>
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <map>
@@ -584,6 +585,43 @@ harp_status_t harp_fast_build(harp_plan *plan) {
         const int64_t co = hi + lo + (sl & 7);
         return phys_in(L, dir == 0 ? (int64_t)plan->h_perm[(size_t)co] : inv[(size_t)co]) + 8 * (sl >> 3);
     };
+    // Stores of the reordering phase.  The four lanes q of a quarter-warp write the slots of the output runs
+    // r = q + 4j in two neighbouring rows.  Starting from the identity, pairs of runs are swapped while that
+    // lowers the number of shared-memory wavefronts (judged on the first item; the other items differ by a
+    // constant offset).  Returns the wavefronts of one item's four store steps (4 = conflict-free) and, if
+    // asked, the assignment.
+    auto reorder_store_wavefronts = [&](const Layout &L, int dir, int64_t pitch_el, int *slot_of_out) {
+        int slot_of[16];
+        for (int r = 0; r < 16; ++r) slot_of[r] = r;
+        int64_t off16[16];
+        for (int sl = 0; sl < 16; ++sl) off16[sl] = reorder_off(L, dir, 0, 0, sl) / 8;
+        auto slot_cost = [&]() {
+            int total = 0;
+            for (int j = 0; j < 4; ++j) {
+                int cnt[8] = {0, 0, 0, 0, 0, 0, 0, 0}, worst = 0;
+                for (int q = 0; q < 4; ++q)
+                    for (int row = 0; row < 2; ++row) {
+                        const int64_t sidx = off16[slot_of[q + 4 * j]] + row * (pitch_el / 8);
+                        worst = std::max(worst, ++cnt[((sidx % 8) + 8) % 8]);
+                    }
+                total += worst;
+            }
+            return total;
+        };
+        int cur = slot_cost();
+        for (bool improved = true; improved && cur > 4;) {
+            improved = false;
+            for (int a = 0; a < 16; ++a)
+                for (int b = a + 1; b < 16; ++b) {
+                    std::swap(slot_of[a], slot_of[b]);
+                    const int c2 = slot_cost();
+                    if (c2 < cur) { cur = c2; improved = true; }
+                    else std::swap(slot_of[a], slot_of[b]);
+                }
+        }
+        if (slot_of_out) for (int r = 0; r < 16; ++r) slot_of_out[r] = slot_of[r];
+        return cur;
+    };
     // scheme 0: plain (both tile copies follow the layout); 1: L is the source-ordered layout of
     // the forward reordering scheme; 2: L is the output-ordered layout of the transpose one
     auto layout_cost = [&](const Layout &L, int scheme) {
@@ -618,6 +656,8 @@ harp_status_t harp_fast_build(harp_plan *plan) {
                 const int64_t o = 8 * c, span = So * Bo;                              // o = hi + lo + r*So
                 return reorder_off(L, scheme - 1, o / span * span, o % So, (int)((o / So) % Bo));
             });
+            // the reordering phase's own stores: 1.0 when conflict-free
+            if (Bo == 16 && So % 8 == 0) cost += 0.25 * reorder_store_wavefronts(L, scheme - 1, pitch_of(L), nullptr);
         } else {
             cost += map_cost([&](int64_t c) { return phys_in(L, 8 * c); });
         }
@@ -760,31 +800,12 @@ harp_status_t harp_fast_build(harp_plan *plan) {
         const Layout &L = dir == 0 ? Lsrc : Lnat;
         const int pr = dir == 0 ? np - 1 : 0;
         const int64_t So = dir == 0 ? phases[(size_t)pr].S : S_src[(size_t)pr], span = So * phases[(size_t)pr].B;
-        // The four lanes q of a quarter-warp access the slots of r = q + 4j in two neighbouring
-        // rows.  Starting from the identity, swap pairs while that lowers the number of
-        // shared-memory wavefronts (judged on the first item; the other items differ by a
-        // constant offset).
         int slot_of[16];
-        for (int r = 0; r < 16; ++r) slot_of[r] = r;
-        auto slot_cost = [&]() {
-            int total = 0;
-            for (int j = 0; j < 4; ++j) {
-                std::vector<int64_t> slots;
-                for (int q = 0; q < 4; ++q)
-                    for (int row = 0; row < 2; ++row) slots.push_back(reorder_off(L, dir, 0, 0, slot_of[q + 4 * j]) / 8 + row * (pitch / 8));
-                total += worst_bank(slots);
-            }
-            return total;
-        };
-        for (bool improved = true; improved;) {
-            improved = false;
-            for (int a = 0; a < 16; ++a)
-                for (int b = a + 1; b < 16; ++b) {
-                    const int before = slot_cost();
-                    std::swap(slot_of[a], slot_of[b]);
-                    if (slot_cost() < before) improved = true;
-                    else std::swap(slot_of[a], slot_of[b]);
-                }
+        const int store_wavefronts = reorder_store_wavefronts(L, dir, pitch, slot_of);
+        if (getenv("HARP_DEBUG_LAYOUT")) {
+            fprintf(stderr, "dir %d: reorder-phase store wavefronts per item %d (ideal 4); W =", dir, store_wavefronts);
+            for (int p = 0; p < np; ++p) fprintf(stderr, " (%lld,%lld,%d)", (long long)L.W[(size_t)p], (long long)L.gp[(size_t)p], L.lm[(size_t)p]);
+            fprintf(stderr, " pitch %lld\n", (long long)pitch);
         }
         chunk_out[dir].assign((size_t)(d / 8), 0);
         for (int64_t hi = 0; hi < d; hi += span)
